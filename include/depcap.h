@@ -1,0 +1,247 @@
+/*
+ * depcap.h — C ABI of the DepCap block-step library (CUDA, sm_100a).
+ *
+ * One call of dc_step runs one block-wise denoising step of a masked diffusion LM on one GPU:
+ * the bidirectional transformer forward that re-predicts the candidate window over a cached
+ * clean context, fused with the per-step signals DepCap decides on, and the block-boundary
+ * decision.  dc_select then picks the conflict-free subset of tokens to commit.
+ *
+ * Paper: "DepCap: Adaptive Block-Wise Parallel Decoding for Efficient Diffusion LM Inference".
+ * Passages each call follows are cited at the call.  Notation follows the paper:
+ *   B        the last decoded block (length Lb), c the decoded context before it
+ *   window   the L_window = min(L_max, L_remain) candidate positions after the frontier
+ *   p_curr   p(Z_k | c, b): prediction with the last block decoded      (Section 4.2 / 4.4)
+ *   p_prev   p(Z_k | c):    prediction with the last block still masked
+ *   I_k      KL(p_curr || p_prev), last-block influence                  (Eq. 3)
+ *   H_k      entropy of p_curr                                           (Section 4.2)
+ *   S_k      I~_k - lambda * H~_k, dependency score                      (Eq. 4)
+ *   c_i      max_v p_i(v), confidence; yhat_i its argmax                 (Section 4.3)
+ *   D_ij     log p_i(yhat_j) + log p_j(yhat_i), conflict score           (Eq. 6)
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the GPU that was current in dc_create;
+ *     "host" pointers are ordinary host memory read during the call.
+ *   - All buffers are owned by the caller.  The library allocates only its own workspace, in
+ *     dc_create, and frees it in dc_destroy.  Weight and cache pointers are borrowed: they must
+ *     stay valid and unchanged while a call that reads them is in flight.
+ *   - dc_step / dc_select / dc_boundary only enqueue work on the context's stream and return;
+ *     outputs are valid after the caller synchronises that stream.
+ *   - Every call returns a dc_status.  Argument and shape errors are detected on the host before
+ *     anything is launched and leave the outputs untouched; dc_last_error gives the reason.
+ *     Conditions detected on the device (an expired bounded wait) are written to status[b].
+ *   - Calls on one context are not thread-safe.
+ *   - Matrix layouts are row-major; weights are [out_features, in_features].
+ *   - Element type of weights, caches and h_final_in is dc_config.dtype (fp32 or bf16).  In the
+ *     bf16 path every GEMM input is rounded to bf16, accumulation and the residual stream are fp32.
+ */
+#ifndef DEPCAP_H_
+#define DEPCAP_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DC_API __attribute__((visibility("default")))
+#else
+#define DC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dc_status {
+  DC_OK = 0,
+  DC_ERR_INVALID_ARG = 1, /* null pointer, bad enum value, negative size                    */
+  DC_ERR_SHAPE = 2,       /* a length exceeds the capacity given to dc_create               */
+  DC_ERR_UNSUPPORTED = 3, /* a shape the kernels cannot handle (see dc_create)              */
+  DC_ERR_NOMEM = 4,       /* workspace allocation failed                                    */
+  DC_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                            */
+  DC_ERR_TIMEOUT = 6,     /* device side: a bounded wait inside a kernel ran out            */
+  DC_ERR_INDEX = 7        /* device side: a token id outside [0, vocab)                     */
+} dc_status;
+
+enum { DC_F32 = 0, DC_BF16 = 1 };                       /* dc_config.dtype             */
+enum { DC_NORM_MAX = 0, DC_NORM_MINMAX = 1, DC_NORM_NONE = 2 };   /* dc_config.norm_mode */
+enum { DC_BOUNDARY_FIRST_NEG = 0, DC_BOUNDARY_CUMULATIVE = 1 };   /* dc_config.boundary_mode */
+enum { DC_CAP_LITERAL = 0, DC_CAP_STRICT = 1 };                   /* dc_config.cap_mode  */
+enum { DC_IMPL_AUTO = 0, DC_IMPL_SIMT = 1 };                      /* dc_config.impl      */
+enum { DC_MAX_BATCH = 32, DC_MAX_WINDOW = 256 };
+
+/* dc_step_in.flags */
+enum {
+  DC_STEP_INFLUENCE = 1, /* also run the prev variant and reduce I_k (Eq. 3)                */
+  DC_STEP_BOUNDARY = 2   /* run the boundary rule (Section 4.2) and write block_len         */
+};
+
+typedef struct dc_config {
+  /* backbone shape (the paper treats the DLM as given; these name it) */
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+  int32_t mask_id;   /* id of [MASK] (Section 3)                                            */
+  int32_t dtype;     /* DC_F32 | DC_BF16                                                    */
+  float rms_eps;     /* RMSNorm epsilon                                                     */
+  float rope_theta;  /* rotary base; pairs (i, i + head_dim/2), angle pos * theta^(-2i/hd)  */
+  /* capacities: fix the layouts of caches and outputs */
+  int32_t max_batch;  /* <= DC_MAX_BATCH                                                    */
+  int32_t max_ctx;    /* multiple of 64                                                     */
+  int32_t max_last;   /* longest last decoded block                                         */
+  int32_t max_window; /* <= DC_MAX_WINDOW, multiple of 16                                   */
+  /* DepCap hyper-parameters ("Hyperparameter settings": 1.2, 8, 128, 0.8, 0.95, -16.0)     */
+  float lambda;
+  int32_t L_min, L_max;
+  float tau_low, tau_high, gamma;
+  /* readings of points the paper leaves open */
+  int32_t smooth_radius;    /* centered moving average over 2r+1 in-range taps; 0 = off     */
+  int32_t norm_mode;        /* how I and H are normalised inside the window                 */
+  int32_t boundary_mode;    /* first S_k < 0 (Section 4.2) or first negative running sum    */
+                            /* of S_k (the cumulative criterion of Section 4.4)             */
+  int32_t cap_mode;         /* Algorithm 1 as printed, or phase 1 also conflict-checked     */
+  int32_t forbid_mask_pred; /* 1: [MASK] is removed from the softmax of both variants       */
+  int32_t impl;             /* DC_IMPL_AUTO: tensor-core kernels where the shape allows;     */
+                            /* DC_IMPL_SIMT: plain CUDA-core kernels only (any shape)       */
+} dc_config;
+
+/* Borrowed device pointers.  Per-layer members are HOST arrays of n_layers device pointers. */
+typedef struct dc_weights {
+  const void* embed;          /* [vocab, d_model]                                           */
+  const void* const* wq;      /* [n_q_heads*head_dim, d_model]                              */
+  const void* const* wk;      /* [n_kv_heads*head_dim, d_model]                             */
+  const void* const* wv;      /* [n_kv_heads*head_dim, d_model]                             */
+  const void* const* wo;      /* [d_model, n_q_heads*head_dim]                              */
+  const void* const* w_gate;  /* [d_ff, d_model]                                            */
+  const void* const* w_up;    /* [d_ff, d_model]                                            */
+  const void* const* w_down;  /* [d_model, d_ff]                                            */
+  const void* const* norm1;   /* [d_model] gain of the pre-attention RMSNorm                */
+  const void* const* norm2;   /* [d_model] gain of the pre-MLP RMSNorm                      */
+  const void* final_norm;     /* [d_model]                                                  */
+  const void* lm_head;        /* [vocab, d_model] (untied)                                  */
+} dc_weights;
+
+typedef struct dc_step_in {
+  int32_t batch; /* sequences in this step, 1..max_batch; sequence b uses cache slot b      */
+  int32_t flags; /* DC_STEP_*                                                                */
+  /* context cache, device, read-only.  K is stored rotated (post-RoPE).
+   *   k_cache [n_layers][max_batch][n_kv_heads][max_ctx][head_dim]
+   *   v_cache [n_layers][max_batch][n_kv_heads][head_dim][max_ctx]   (V transposed: keys are
+   *           the contiguous axis, which is what the PV product streams)
+   * Only the first ctx_len[b] keys of slot b are read; the rest may hold anything.
+   * Both may be null when every ctx_len is 0. */
+  const void* k_cache;
+  const void* v_cache;
+  const int32_t* ctx_len;    /* host [batch], 0..max_ctx                                    */
+  const int32_t* last_ids;   /* device [batch][max_last]: the last decoded block B          */
+  const int32_t* last_len;   /* host [batch], 0..max_last; 0 = no last block (cold start)   */
+  const int32_t* win_ids;    /* device [batch][max_window]; mask_id = still masked          */
+  const int32_t* win_len;    /* host [batch], 1..max_window: window positions supplied      */
+  const int32_t* remain_len; /* host [batch]: L_remain, masked tokens after the frontier    */
+  /* Optional, device, [batch][2][max_window][d_model] (curr, prev): replaces the transformer
+   * stack's output as the LM-head input (the stack still runs).  For tests and benchmarks that
+   * need shaped distributions from random-init weights.  Null in normal use. */
+  const void* h_final_in;
+} dc_step_in;
+
+/* Caller-owned device buffers; rows b >= batch and columns k >= win_len[b] are not written.
+ * Any pointer except status may be null to skip that output. */
+typedef struct dc_step_out {
+  int32_t* pred_id;     /* [batch][max_window] yhat_k                                       */
+  float* conf;          /* [batch][max_window] c_k = max_v p_curr(v)                        */
+  float* entropy;       /* [batch][max_window] H_k                                          */
+  float* influence;     /* [batch][max_window] I_k (0 without a prev variant)               */
+  float* lse;           /* [batch][max_window] log-sum-exp of the curr logits               */
+  float* xlogp;         /* [batch][max_window][max_window] log p_i(yhat_j)  (Eq. 6 halves)  */
+  float* score;         /* [batch][max_window] S_k                (DC_STEP_BOUNDARY)        */
+  float* cum_influence; /* [batch][max_window] sum_{j<=k} I_j     (DC_STEP_BOUNDARY)        */
+  float* cum_score;     /* [batch][max_window] sum_{j<=k} S_j     (DC_STEP_BOUNDARY)        */
+  int32_t* block_len;   /* [batch] next block length L            (DC_STEP_BOUNDARY)        */
+  int32_t* status;      /* [batch] DC_OK or a device-side dc_status; required               */
+} dc_step_out;
+
+typedef struct dc_boundary_in {
+  int32_t batch;
+  const float* influence;    /* device [batch][max_window]                                  */
+  const float* entropy;      /* device [batch][max_window]                                  */
+  const int32_t* win_len;    /* host [batch]                                                */
+  const int32_t* remain_len; /* host [batch]                                                */
+  const int32_t* have_prev;  /* host [batch]; 0 = cold start (L = L_min)                    */
+} dc_boundary_in;
+
+typedef struct dc_boundary_out {
+  float* score;         /* device [batch][max_window], may be null                          */
+  float* cum_influence; /* device [batch][max_window], may be null                          */
+  float* cum_score;     /* device [batch][max_window], may be null                          */
+  int32_t* block_len;   /* device [batch], required                                         */
+} dc_boundary_out;
+
+typedef struct dc_select_in {
+  int32_t batch;
+  const float* conf;        /* device [batch][max_window]                                   */
+  const int32_t* win_ids;   /* device [batch][max_window]; candidates are == mask_id        */
+  const float* xlogp;       /* device [batch][max_window][max_window]                       */
+  const int32_t* block_len; /* device [batch]: the current block is window[0, block_len)    */
+  const int32_t* win_len;   /* host [batch]                                                 */
+  int32_t override_thresholds; /* 1: use the three values below instead of the config's     */
+  float tau_low, tau_high, gamma;
+} dc_select_in;
+
+typedef struct dc_select_out {
+  uint8_t* sel_mask;  /* device [batch][max_window] 1 = commit this position                */
+  int32_t* sel_idx;   /* device [batch][max_window] selected positions, ascending           */
+  int32_t* sel_count; /* device [batch] |S|                                                 */
+} dc_select_out;
+
+typedef struct dc_ctx dc_ctx; /* opaque */
+
+/* Create a context: validates the configuration, records the (borrowed) weight pointers, and
+ * allocates the workspace for the given capacities on the current CUDA device.
+ * cuda_stream: a cudaStream_t (null = the legacy default stream); all work is ordered on it.
+ * Tensor-core kernels need dtype bf16, head_dim 128, d_model and d_ff multiples of 128; any
+ * other shape runs on the CUDA-core kernels.  Errors: INVALID_ARG, UNSUPPORTED, NOMEM, CUDA.
+ * The backbone is the pre-norm transformer the paper's backbones share (Section 5.1). */
+DC_API int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_ctx** out);
+
+/* One block-step (Section 3, Eq. 1-2: predictions for the masked positions of the active block
+ * given the decoded context; Section 4.2, Eq. 3-4: I_k, H_k, S_k and the block boundary).
+ * Rows fed to the backbone per sequence: the last decoded block followed by the window, at
+ * absolute positions ctx_len[b] + r; with DC_STEP_INFLUENCE a second variant with the last
+ * block's ids replaced by mask_id runs in the same pass (p_prev).  Every active row attends all
+ * ctx_len[b] cached keys and all active rows of its own variant (no causal mask).
+ * Errors: INVALID_ARG, SHAPE, CUDA (host side); status[b] (device side). */
+DC_API int dc_step(dc_ctx* ctx, const dc_step_in* in, const dc_step_out* out);
+
+/* The boundary rule alone on caller-supplied signals (Section 4.2; cumulative form Section 4.4):
+ * smooth, normalise, S_k = I~_k - lambda*H~_k, first negative, clip to [L_min, L_window].
+ * dc_step runs the same kernel when DC_STEP_BOUNDARY is set. */
+DC_API int dc_boundary(dc_ctx* ctx, const dc_boundary_in* in, const dc_boundary_out* out);
+
+/* CAP-Decoding (Section 4.3, Eq. 5-6, Algorithm 1): candidate pool, pairwise conflicts,
+ * high-confidence phase, greedy completion, single-token fallback.  Reads the buffers a
+ * previous dc_step wrote (or any caller-made ones). */
+DC_API int dc_select(dc_ctx* ctx, const dc_select_in* in, const dc_select_out* out);
+
+/* Frees the workspace.  The caller must have synchronised the stream.  Null is a no-op. */
+DC_API int dc_destroy(dc_ctx* ctx);
+
+/* Human-readable reason for the last non-OK return on this context (never null).  With a null
+ * context: the reason for the last failed dc_create on this thread. */
+DC_API const char* dc_last_error(const dc_ctx* ctx);
+
+/* Debug: copies the curr-variant (variant 0) or prev-variant (1) logits of the last dc_step into
+ * out [batch][max_window][vocab] fp32 (device).  Only available when the CUDA-core LM head ran
+ * (DC_IMPL_SIMT or an fp32 model); otherwise DC_ERR_UNSUPPORTED.  No paper counterpart. */
+DC_API int dc_debug_logits(dc_ctx* ctx, int32_t variant, float* out);
+
+/* Per-stage device time of the last dc_step_profiled call, in milliseconds. */
+enum { DC_STAGE_EMBED = 0, DC_STAGE_NORM, DC_STAGE_QKV, DC_STAGE_ATTN, DC_STAGE_OPROJ,
+       DC_STAGE_GATEUP, DC_STAGE_DOWN, DC_STAGE_LMHEAD, DC_STAGE_XLOGP, DC_STAGE_BOUNDARY,
+       DC_STAGE_COUNT };
+
+/* dc_step with CUDA events around every stage; synchronises the stream before returning and
+ * fills stage_ms[DC_STAGE_COUNT] (host) with the summed device time per stage and
+ * stage_launches[DC_STAGE_COUNT] (host) with the kernel launches per stage.  For measurement;
+ * same results as dc_step.  No paper counterpart. */
+DC_API int dc_step_profiled(dc_ctx* ctx, const dc_step_in* in, const dc_step_out* out, float* stage_ms,
+                     int32_t* stage_launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEPCAP_H_ */

@@ -1,0 +1,323 @@
+"""ctypes binding of include/depcap.h.  Same names, same argument meaning; torch tensors are used
+only as device/host buffers and for the CUDA stream."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdepcap.so")
+
+DC_OK = 0
+DC_F32, DC_BF16 = 0, 1
+DC_STEP_INFLUENCE, DC_STEP_BOUNDARY = 1, 2
+DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
+STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
+               "boundary"]
+EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
+           "dc_debug_logits", "dc_step_profiled"]
+
+
+class DepCapError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"depcap error {code}: {msg}")
+        self.code = code
+
+
+class dc_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ff", "vocab",
+                 "mask_id", "dtype")] + \
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
+               [(n, C.c_int32) for n in ("max_batch", "max_ctx", "max_last", "max_window")] + \
+               [("lambda_", C.c_float), ("L_min", C.c_int32), ("L_max", C.c_int32),
+                ("tau_low", C.c_float), ("tau_high", C.c_float), ("gamma", C.c_float)] + \
+               [(n, C.c_int32) for n in ("smooth_radius", "norm_mode", "boundary_mode",
+                                         "cap_mode", "forbid_mask_pred", "impl")]
+
+
+_PP = C.POINTER(C.c_void_p)
+
+
+class dc_weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p)] + \
+               [(n, _PP) for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm1",
+                                   "norm2")] + \
+               [("final_norm", C.c_void_p), ("lm_head", C.c_void_p)]
+
+
+_I32P = C.POINTER(C.c_int32)
+
+
+class dc_step_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("flags", C.c_int32), ("k_cache", C.c_void_p),
+                ("v_cache", C.c_void_p), ("ctx_len", _I32P), ("last_ids", C.c_void_p),
+                ("last_len", _I32P), ("win_ids", C.c_void_p), ("win_len", _I32P),
+                ("remain_len", _I32P), ("h_final_in", C.c_void_p)]
+
+
+class dc_step_out(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("pred_id", "conf", "entropy", "influence", "lse", "xlogp", "score",
+                 "cum_influence", "cum_score", "block_len", "status")]
+
+
+class dc_boundary_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("influence", C.c_void_p), ("entropy", C.c_void_p),
+                ("win_len", _I32P), ("remain_len", _I32P), ("have_prev", _I32P)]
+
+
+class dc_boundary_out(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("score", "cum_influence", "cum_score", "block_len")]
+
+
+class dc_select_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("conf", C.c_void_p), ("win_ids", C.c_void_p),
+                ("xlogp", C.c_void_p), ("block_len", C.c_void_p), ("win_len", _I32P),
+                ("override_thresholds", C.c_int32), ("tau_low", C.c_float),
+                ("tau_high", C.c_float), ("gamma", C.c_float)]
+
+
+class dc_select_out(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("sel_mask", "sel_idx", "sel_count")]
+
+
+_lib = None
+
+
+def load_library(path: str | None = None):
+    """Loads libdepcap.so (built in-tree by build.py).  Fails loudly when it is missing: there
+    is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(f"{p} not found: run `python -m paper_2604_15750_b200.build` "
+                          "(or __graft_entry__.build()) first; there is no fallback path")
+    lib_ = C.CDLL(p)
+    lib_.dc_create.argtypes = [C.POINTER(dc_config), C.POINTER(dc_weights), C.c_void_p,
+                               C.POINTER(C.c_void_p)]
+    lib_.dc_step.argtypes = [C.c_void_p, C.POINTER(dc_step_in), C.POINTER(dc_step_out)]
+    lib_.dc_step_profiled.argtypes = [C.c_void_p, C.POINTER(dc_step_in), C.POINTER(dc_step_out),
+                                      C.POINTER(C.c_float), _I32P]
+    lib_.dc_boundary.argtypes = [C.c_void_p, C.POINTER(dc_boundary_in),
+                                 C.POINTER(dc_boundary_out)]
+    lib_.dc_select.argtypes = [C.c_void_p, C.POINTER(dc_select_in), C.POINTER(dc_select_out)]
+    lib_.dc_destroy.argtypes = [C.c_void_p]
+    lib_.dc_debug_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+    lib_.dc_last_error.argtypes = [C.c_void_p]
+    lib_.dc_last_error.restype = C.c_char_p
+    for n in EXPORTS:
+        if n != "dc_last_error":
+            getattr(lib_, n).restype = C.c_int
+    if path is None:
+        _lib = lib_
+    return lib_
+
+
+def lib():
+    return load_library()
+
+
+@dataclass
+class Hyper:
+    """DepCap hyper-parameters (defaults of the paper's experimental settings) and the
+    selectors for the points the paper leaves open."""
+    lam: float = 1.2
+    L_min: int = 8
+    L_max: int = 128
+    tau_low: float = 0.8
+    tau_high: float = 0.95
+    gamma: float = -16.0
+    smooth_radius: int = 1
+    norm_mode: int = 0
+    boundary_mode: int = 0
+    cap_mode: int = 0
+    forbid_mask_pred: bool = True
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _host_i32(values, n):
+    arr = (C.c_int32 * n)(*[int(v) for v in values])
+    return arr
+
+
+def pack_kv_cache(k_logical: torch.Tensor, v_logical: torch.Tensor, max_batch: int, max_ctx: int):
+    """Logical caches [layers, batch, n_kv, ctx, hd] -> the library's layouts:
+    K [layers, max_batch, n_kv, max_ctx, hd], V [layers, max_batch, n_kv, hd, max_ctx]."""
+    L, B, H, P, D = k_logical.shape
+    k = torch.zeros((L, max_batch, H, max_ctx, D), dtype=k_logical.dtype, device=k_logical.device)
+    v = torch.zeros((L, max_batch, H, D, max_ctx), dtype=v_logical.dtype, device=v_logical.device)
+    k[:, :B, :, :P, :] = k_logical
+    v[:, :B, :, :, :P] = v_logical.transpose(3, 4)
+    return k, v
+
+
+class DepCap:
+    """One dc_ctx plus reusable output buffers.  `weights` is the dict made by
+    inputs.make_weights (tensors already on the CUDA device, dtype = model dtype)."""
+
+    def __init__(self, *, n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab, mask_id,
+                 dtype, weights, max_batch, max_ctx, max_last, max_window, hyper: Hyper = Hyper(),
+                 rms_eps=1e-5, rope_theta=10000.0, impl=DC_IMPL_AUTO, stream=None):
+        self._lib = lib()
+        self._ctx = C.c_void_p()
+        if not torch.cuda.is_available():
+            raise RuntimeError("DepCap needs a CUDA device; there is no CPU path")
+        self.device = weights["embed"].device
+        assert self.device.type == "cuda"
+        self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        self.max_batch, self.max_ctx = max_batch, max_ctx
+        self.max_last, self.max_window = max_last, max_window
+        self.vocab, self.d_model, self.mask_id = vocab, d_model, mask_id
+        self.stream = stream or torch.cuda.current_stream(self.device)
+        cfg = dc_config(n_layers=n_layers, d_model=d_model, n_q_heads=n_q_heads,
+                        n_kv_heads=n_kv_heads, head_dim=head_dim, d_ff=d_ff, vocab=vocab,
+                        mask_id=mask_id, dtype=DC_F32 if dtype == "f32" else DC_BF16,
+                        rms_eps=rms_eps, rope_theta=rope_theta, max_batch=max_batch,
+                        max_ctx=max_ctx, max_last=max_last, max_window=max_window,
+                        lambda_=hyper.lam, L_min=hyper.L_min, L_max=hyper.L_max,
+                        tau_low=hyper.tau_low, tau_high=hyper.tau_high, gamma=hyper.gamma,
+                        smooth_radius=hyper.smooth_radius, norm_mode=hyper.norm_mode,
+                        boundary_mode=hyper.boundary_mode, cap_mode=hyper.cap_mode,
+                        forbid_mask_pred=int(hyper.forbid_mask_pred), impl=impl)
+        self._weights = weights          # keep the borrowed tensors alive
+        layers = weights["layers"][:n_layers]
+        for t in [weights["embed"], weights["lm_head"], weights["final_norm"]] + \
+                 [t for lw in layers for t in lw.values()]:
+            assert t.is_cuda and t.is_contiguous() and t.dtype == self.tdtype
+        w = dc_weights(embed=_ptr(weights["embed"]), final_norm=_ptr(weights["final_norm"]),
+                       lm_head=_ptr(weights["lm_head"]))
+        self._arrays = []
+        for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm1", "norm2"):
+            arr = (C.c_void_p * max(n_layers, 1))(*[lw[name].data_ptr() for lw in layers])
+            self._arrays.append(arr)
+            setattr(w, name, C.cast(arr, _PP))
+        with torch.cuda.device(self.device):
+            rc = self._lib.dc_create(C.byref(cfg), C.byref(w), C.c_void_p(self.stream.cuda_stream),
+                                     C.byref(self._ctx))
+        if rc != DC_OK:
+            raise DepCapError(rc, self._lib.dc_last_error(None).decode())
+        B, W = max_batch, max_window
+        dev = self.device
+        f = lambda *s: torch.zeros(s, dtype=torch.float32, device=dev)
+        i = lambda *s: torch.zeros(s, dtype=torch.int32, device=dev)
+        self.out = dict(pred_id=i(B, W), conf=f(B, W), entropy=f(B, W), influence=f(B, W),
+                        lse=f(B, W), xlogp=f(B, W, W), score=f(B, W), cum_influence=f(B, W),
+                        cum_score=f(B, W), block_len=i(B), status=i(B))
+        self.sel = dict(sel_mask=torch.zeros((B, W), dtype=torch.uint8, device=dev),
+                        sel_idx=i(B, W), sel_count=i(B))
+
+    @classmethod
+    def from_workload(cls, wl, weights, n_layers=None, hyper=Hyper(), impl=DC_IMPL_AUTO,
+                      max_batch=None, max_ctx=None, max_window=None, max_last=None):
+        r64 = lambda v: (v + 63) // 64 * 64
+        r16 = lambda v: (v + 15) // 16 * 16
+        return cls(n_layers=wl.n_layers if n_layers is None else n_layers, d_model=wl.d_model,
+                   n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                   d_ff=wl.d_ff, vocab=wl.vocab, mask_id=wl.mask_id, dtype=wl.dtype,
+                   weights=weights, max_batch=max_batch or wl.batch,
+                   max_ctx=max_ctx if max_ctx is not None else r64(wl.ctx_max),
+                   max_last=max_last if max_last is not None else wl.last_len,
+                   max_window=max_window or r16(wl.win_len), hyper=hyper, rms_eps=wl.rms_eps,
+                   rope_theta=wl.rope_theta, impl=impl)
+
+    # -- error helper ---------------------------------------------------------------------
+    def _check(self, rc):
+        if rc != DC_OK:
+            raise DepCapError(rc, self._lib.dc_last_error(self._ctx).decode())
+
+    # -- dc_step ---------------------------------------------------------------------------
+    def _step_structs(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len,
+                      remain_len, influence, boundary, h_final, want_xlogp=True):
+        B = len(win_len)
+        self._keep = (k_cache, v_cache, last_ids, win_ids, h_final,
+                      _host_i32(ctx_len, B), _host_i32(last_len, B), _host_i32(win_len, B),
+                      _host_i32(remain_len, B))
+        si = dc_step_in(batch=B, flags=(DC_STEP_INFLUENCE if influence else 0) |
+                        (DC_STEP_BOUNDARY if boundary else 0),
+                        k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                        ctx_len=C.cast(self._keep[5], _I32P), last_ids=_ptr(last_ids),
+                        last_len=C.cast(self._keep[6], _I32P), win_ids=_ptr(win_ids),
+                        win_len=C.cast(self._keep[7], _I32P),
+                        remain_len=C.cast(self._keep[8], _I32P), h_final_in=_ptr(h_final))
+        so = dc_step_out(**{k: _ptr(v) for k, v in self.out.items()})
+        if not want_xlogp:
+            so.xlogp = None
+        return si, so
+
+    def step(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len, remain_len,
+             influence=True, boundary=True, h_final=None):
+        """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled."""
+        si, so = self._step_structs(k_cache, v_cache, ctx_len, last_ids, last_len, win_ids,
+                                    win_len, remain_len, influence, boundary, h_final)
+        self._check(self._lib.dc_step(self._ctx, C.byref(si), C.byref(so)))
+        return self.out
+
+    def step_profiled(self, *args, **kw):
+        si, so = self._step_structs(*args, **kw)
+        ms = (C.c_float * len(STAGE_NAMES))()
+        nl = (C.c_int32 * len(STAGE_NAMES))()
+        self._check(self._lib.dc_step_profiled(self._ctx, C.byref(si), C.byref(so), ms, nl))
+        return {n: float(ms[i]) for i, n in enumerate(STAGE_NAMES)}, \
+               {n: int(nl[i]) for i, n in enumerate(STAGE_NAMES)}
+
+    # -- dc_boundary -----------------------------------------------------------------------
+    def boundary(self, influence, entropy, win_len, remain_len, have_prev=None):
+        B = len(win_len)
+        hp = _host_i32(have_prev if have_prev is not None else [1] * B, B)
+        wl_, rl_ = _host_i32(win_len, B), _host_i32(remain_len, B)
+        bi = dc_boundary_in(batch=B, influence=_ptr(influence), entropy=_ptr(entropy),
+                            win_len=C.cast(wl_, _I32P), remain_len=C.cast(rl_, _I32P),
+                            have_prev=C.cast(hp, _I32P))
+        bo = dc_boundary_out(score=_ptr(self.out["score"]),
+                             cum_influence=_ptr(self.out["cum_influence"]),
+                             cum_score=_ptr(self.out["cum_score"]),
+                             block_len=_ptr(self.out["block_len"]))
+        self._check(self._lib.dc_boundary(self._ctx, C.byref(bi), C.byref(bo)))
+        return self.out
+
+    # -- dc_select -------------------------------------------------------------------------
+    def select(self, win_ids, win_len, conf=None, xlogp=None, block_len=None, thresholds=None):
+        B = len(win_len)
+        wl_ = _host_i32(win_len, B)
+        conf = self.out["conf"] if conf is None else conf
+        xlogp = self.out["xlogp"] if xlogp is None else xlogp
+        block_len = self.out["block_len"] if block_len is None else block_len
+        self._keep_sel = (win_ids, conf, xlogp, block_len, wl_)
+        si = dc_select_in(batch=B, conf=_ptr(conf), win_ids=_ptr(win_ids), xlogp=_ptr(xlogp),
+                          block_len=_ptr(block_len), win_len=C.cast(wl_, _I32P))
+        if thresholds is not None:
+            si.override_thresholds = 1
+            si.tau_low, si.tau_high, si.gamma = thresholds
+        so = dc_select_out(**{k: _ptr(v) for k, v in self.sel.items()})
+        self._check(self._lib.dc_select(self._ctx, C.byref(si), C.byref(so)))
+        return self.sel
+
+    def debug_logits(self, variant=0):
+        out = torch.zeros((self.max_batch, self.max_window, self.vocab), dtype=torch.float32,
+                          device=self.device)
+        self._check(self._lib.dc_debug_logits(self._ctx, variant, _ptr(out)))
+        return out
+
+    def synchronize(self):
+        self.stream.synchronize()
+
+    def close(self):
+        if self._ctx:
+            self.stream.synchronize()
+            self._lib.dc_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

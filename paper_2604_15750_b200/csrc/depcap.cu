@@ -1,0 +1,498 @@
+// C ABI and step scheduler of the DepCap block-step library.
+//
+// The scheduler turns one dc_step into a fixed sequence of kernel launches on the context's
+// stream; it never synchronises (except in dc_step_profiled) and never touches the outputs on
+// an argument error.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "kernels.h"
+#include "tc.h"
+
+using namespace dc;
+
+namespace {
+
+thread_local std::string g_create_error = "";
+
+struct Profiler : dc::StageHook {
+  bool on = false;
+  struct Span { int stage; cudaEvent_t a, b; };
+  std::vector<Span> spans;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  int launches[DC_STAGE_COUNT] = {};
+  cudaStream_t s = nullptr;
+  cudaEvent_t get() {
+    if (used == pool.size()) {
+      cudaEvent_t e;
+      cudaEventCreate(&e);
+      pool.push_back(e);
+    }
+    return pool[used++];
+  }
+  void begin(int stage, int n_launch) override {
+    launches[stage] += n_launch;
+    if (!on) return;
+    Span sp{stage, get(), get()};
+    cudaEventRecord(sp.a, s);
+    spans.push_back(sp);
+  }
+  void end() override {
+    if (!on) return;
+    cudaEventRecord(spans.back().b, s);
+  }
+  void reset(bool enable, cudaStream_t st) {
+    on = enable; s = st; used = 0; spans.clear();
+    memset(launches, 0, sizeof(launches));
+  }
+  ~Profiler() { for (auto e : pool) cudaEventDestroy(e); }
+};
+
+}  // namespace
+
+struct dc_ctx {
+  dc_config cfg{};
+  Hyper hp{};
+  cudaStream_t stream = nullptr;
+  int device = 0;
+  bool bf16 = false;
+  bool use_tc = false;  // tensor-core kernels for the dense layers / LM head / attention
+  const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+  std::vector<const void*> wq, wk, wv, wo, w_gate, w_up, w_down, norm1, norm2;
+  // capacities
+  int R_cap_max = 0, M_max = 0, Mlm_max = 0;
+  // workspace (device)
+  std::vector<void*> allocs;
+  float* x = nullptr;        // residual stream [M, d] fp32
+  void* a = nullptr;         // normed activations [M, d]
+  void* q = nullptr;         // [M, nq*hd] rotated
+  void* k = nullptr;         // [M, nkv*hd] rotated
+  void* v = nullptr;         // [M, nkv*hd]
+  void* o = nullptr;         // attention output [M, nq*hd]
+  void* act = nullptr;       // SwiGLU output [M, F]
+  float* tmp = nullptr;      // fp32 GEMM outputs of the CUDA-core path
+  void* h = nullptr;         // LM-head input [M_lm, d]
+  float* logits = nullptr;   // [M_lm, V] fp32, CUDA-core LM head only
+  float* cos_sin = nullptr;  // RoPE table [max_batch * R_cap_max, hd]
+  int32_t* ws_pred = nullptr;
+  float *ws_conf = nullptr, *ws_ent = nullptr, *ws_infl = nullptr, *ws_lse = nullptr;
+  TcState* tc = nullptr;
+  SeqMeta last_meta{};
+  bool have_logits = false;
+  Profiler prof;
+  std::string err;
+};
+
+namespace {
+
+int fail(dc_ctx* c, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  if (c) c->err = buf; else g_create_error = buf;
+  return code;
+}
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+template <typename T>
+T* ws_alloc(dc_ctx* c, size_t n, bool* ok) {
+  void* p = nullptr;
+  if (n == 0) n = 1;
+  if (cudaMalloc(&p, n * sizeof(T)) != cudaSuccess) {
+    *ok = false;
+    cudaGetLastError();
+    return nullptr;
+  }
+  c->allocs.push_back(p);
+  return reinterpret_cast<T*>(p);
+}
+
+int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const int32_t* last_len,
+               const int32_t* win_len, const int32_t* remain_len, SeqMeta* m) {
+  const dc_config& g = c->cfg;
+  if (batch < 1 || batch > g.max_batch)
+    return fail(c, DC_ERR_SHAPE, "batch %d outside [1, max_batch=%d]", batch, g.max_batch);
+  memset(m, 0, sizeof(*m));
+  m->batch = batch;
+  m->nv = (flags & DC_STEP_INFLUENCE) ? 2 : 1;
+  int maxR = 0, maxW = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int P = ctx_len ? ctx_len[b] : 0, Lb = last_len ? last_len[b] : 0, W = win_len[b];
+    if (P < 0 || P > g.max_ctx)
+      return fail(c, DC_ERR_SHAPE, "ctx_len[%d]=%d outside [0, max_ctx=%d]", b, P, g.max_ctx);
+    if (Lb < 0 || Lb > g.max_last)
+      return fail(c, DC_ERR_SHAPE, "last_len[%d]=%d outside [0, max_last=%d]", b, Lb, g.max_last);
+    if (W < 1 || W > g.max_window)
+      return fail(c, DC_ERR_SHAPE, "win_len[%d]=%d outside [1, max_window=%d]", b, W,
+                  g.max_window);
+    m->ctx_len[b] = P; m->last_len[b] = Lb; m->win_len[b] = W;
+    m->remain[b] = remain_len ? remain_len[b] : W;
+    m->have_prev[b] = (m->nv == 2 && Lb > 0) ? 1 : 0;
+    maxR = maxR > Lb + W ? maxR : Lb + W;
+    maxW = maxW > W ? maxW : W;
+  }
+  m->R_cap = round_up(maxR, 16);
+  m->W_cap = round_up(maxW, 16);
+  const int npos = batch * m->W_cap;
+  m->G = npos < 128 ? npos : 128;
+  m->npos_pad = round_up(npos, m->G);
+  return DC_OK;
+}
+
+#define DC_CHECK_LAUNCH(c)                                                                   \
+  do {                                                                                       \
+    cudaError_t e_ = cudaGetLastError();                                                     \
+    if (e_ != cudaSuccess)                                                                   \
+      return fail(c, DC_ERR_CUDA, "CUDA error after launch (%s:%d): %s", __FILE__, __LINE__, \
+                  cudaGetErrorString(e_));                                                   \
+  } while (0)
+
+template <typename T>
+int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqMeta& m) {
+  const dc_config& g = c->cfg;
+  cudaStream_t s = c->stream;
+  Profiler& pf = c->prof;
+  const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
+  const int M = m.nv * m.batch * m.R_cap;
+  const int Mlm = m.nv * m.npos_pad;
+  const int nqkv = (nq + 2 * nkv) * hd;
+  T* a = (T*)c->a; T* q = (T*)c->q; T* k = (T*)c->k; T* v = (T*)c->v; T* o = (T*)c->o;
+  T* act = (T*)c->act; T* h = (T*)c->h;
+  const size_t k_layer = (size_t)g.max_batch * nkv * g.max_ctx * hd;
+
+  cudaMemsetAsync(out->status, 0, sizeof(int32_t) * m.batch, s);
+  pf.begin(DC_STAGE_EMBED, 2);
+  launch_embed<T>((const T*)c->embed, in->last_ids, in->win_ids, g.max_last, g.max_window,
+                  g.mask_id, g.vocab, d, m, c->x, out->status, s);
+  launch_rope_table(m, hd, g.rope_theta, c->cos_sin, s);
+  pf.end();
+  DC_CHECK_LAUNCH(c);
+
+  // split-K partial sums produced by the previous residual GEMM, folded in by the next norm
+  const float* part = nullptr;
+  int nsplit = 0;
+  size_t part_stride = 0;
+
+  for (int l = 0; l < g.n_layers; ++l) {
+    pf.begin(DC_STAGE_NORM, 1);
+    launch_rmsnorm<T>(c->x, part, nsplit, part_stride, (const T*)c->norm1[l], g.rms_eps, M, d, a, s);
+    pf.end();
+    part = nullptr; nsplit = 0;
+    const T* kc = in->k_cache ? (const T*)in->k_cache + (size_t)l * k_layer : nullptr;
+    const T* vc = in->v_cache ? (const T*)in->v_cache + (size_t)l * k_layer : nullptr;
+    if (c->use_tc) {
+      int rc = tc_layer(c->tc, l, m, c->x, (const __nv_bfloat16*)a, (const __nv_bfloat16*)kc,
+                        (const __nv_bfloat16*)vc, c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
+                        &part, &nsplit, &part_stride, pf);
+      if (rc != DC_OK) return fail(c, rc, "tensor-core layer %d failed: %s", l, tc_error(c->tc));
+      continue;
+    }
+    pf.begin(DC_STAGE_QKV, 4);
+    launch_gemm_simt<T>(a, (const T*)c->wq[l], c->tmp, M, nq * hd, d, nqkv, EPI_STORE_F32, s);
+    launch_gemm_simt<T>(a, (const T*)c->wk[l], c->tmp + nq * hd, M, nkv * hd, d, nqkv,
+                        EPI_STORE_F32, s);
+    launch_gemm_simt<T>(a, (const T*)c->wv[l], c->tmp + (nq + nkv) * hd, M, nkv * hd, d, nqkv,
+                        EPI_STORE_F32, s);
+    launch_rope_store<T>(c->tmp, c->cos_sin, m, nq, nkv, hd, q, k, v, s);
+    pf.end();
+    pf.begin(DC_STAGE_ATTN, 1);
+    launch_attn_simt<T>(q, k, v, kc, vc, g.max_ctx, m, nq, nkv, hd, o, s);
+    pf.end();
+    pf.begin(DC_STAGE_OPROJ, 1);
+    launch_gemm_simt<T>(o, (const T*)c->wo[l], c->x, M, d, nq * hd, d, EPI_ADD_F32, s);
+    pf.end();
+    pf.begin(DC_STAGE_NORM, 1);
+    launch_rmsnorm<T>(c->x, nullptr, 0, 0, (const T*)c->norm2[l], g.rms_eps, M, d, a, s);
+    pf.end();
+    pf.begin(DC_STAGE_GATEUP, 3);
+    launch_gemm_simt<T>(a, (const T*)c->w_gate[l], c->tmp, M, F, d, 2 * F, EPI_STORE_F32, s);
+    launch_gemm_simt<T>(a, (const T*)c->w_up[l], c->tmp + F, M, F, d, 2 * F, EPI_STORE_F32, s);
+    launch_swiglu<T>(c->tmp, M, F, act, s);
+    pf.end();
+    pf.begin(DC_STAGE_DOWN, 1);
+    launch_gemm_simt<T>(act, (const T*)c->w_down[l], c->x, M, d, F, d, EPI_ADD_F32, s);
+    pf.end();
+    DC_CHECK_LAUNCH(c);
+  }
+
+  pf.begin(DC_STAGE_NORM, in->h_final_in ? 2 : 1);
+  launch_final_norm<T>(c->x, part, nsplit, part_stride, (const T*)c->final_norm, g.rms_eps, d, m,
+                       h, s);
+  if (in->h_final_in) launch_h_override<T>((const T*)in->h_final_in, g.max_window, d, m, h, s);
+  pf.end();
+
+  SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, g.max_window};
+  if (c->use_tc) {
+    pf.begin(DC_STAGE_LMHEAD, 2);
+    int rc = tc_lmhead(c->tc, m, (const __nv_bfloat16*)h, g.mask_id, g.forbid_mask_pred,
+                       c->ws_pred, c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so);
+    pf.end();
+    if (rc != DC_OK) return fail(c, rc, "tensor-core LM head failed: %s", tc_error(c->tc));
+    c->have_logits = false;
+  } else {
+    pf.begin(DC_STAGE_LMHEAD, 2);
+    launch_gemm_simt<T>(h, (const T*)c->lm_head, c->logits, Mlm, g.vocab, d, g.vocab,
+                        EPI_STORE_F32, s);
+    launch_signals_from_logits(c->logits, g.vocab, g.mask_id, g.forbid_mask_pred, m, c->ws_pred,
+                               c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so, s);
+    pf.end();
+    c->have_logits = true;
+  }
+  if (out->xlogp) {
+    pf.begin(DC_STAGE_XLOGP, 1);
+    launch_xlogp<T>(h, (const T*)c->lm_head, c->ws_pred, c->ws_lse, d, m, g.max_window,
+                    out->xlogp, s);
+    pf.end();
+  }
+  if ((in->flags & DC_STEP_BOUNDARY) && out->block_len) {
+    pf.begin(DC_STAGE_BOUNDARY, 1);
+    launch_boundary(c->ws_infl, c->ws_ent, m.W_cap, m, c->hp, g.max_window, out->score,
+                    out->cum_influence, out->cum_score, out->block_len, s);
+    pf.end();
+  }
+  DC_CHECK_LAUNCH(c);
+  c->last_meta = m;
+  return DC_OK;
+}
+
+int validate_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, SeqMeta* m) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !out) return fail(c, DC_ERR_INVALID_ARG, "null in/out");
+  if (!out->status) return fail(c, DC_ERR_INVALID_ARG, "out->status is required");
+  if (!in->win_ids || !in->win_len) return fail(c, DC_ERR_INVALID_ARG, "win_ids/win_len null");
+  if (in->flags & ~(DC_STEP_INFLUENCE | DC_STEP_BOUNDARY))
+    return fail(c, DC_ERR_INVALID_ARG, "unknown flag bits 0x%x", in->flags);
+  int rc = build_meta(c, in->batch, in->flags, in->ctx_len, in->last_len, in->win_len,
+                      in->remain_len, m);
+  if (rc != DC_OK) return rc;
+  bool any_ctx = false, any_last = false;
+  for (int b = 0; b < m->batch; ++b) {
+    any_ctx |= m->ctx_len[b] > 0;
+    any_last |= m->last_len[b] > 0;
+  }
+  if (any_ctx && (!in->k_cache || !in->v_cache))
+    return fail(c, DC_ERR_INVALID_ARG, "ctx_len > 0 but k_cache/v_cache null");
+  if (any_last && !in->last_ids) return fail(c, DC_ERR_INVALID_ARG, "last_len > 0 but last_ids null");
+  return DC_OK;
+}
+
+int do_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, bool profile,
+            float* stage_ms, int32_t* stage_launches) {
+  SeqMeta m;
+  int rc = validate_step(c, in, out, &m);
+  if (rc != DC_OK) return rc;
+  int dev = -1;
+  cudaGetDevice(&dev);
+  if (dev != c->device) cudaSetDevice(c->device);
+  c->prof.reset(profile, c->stream);
+  rc = c->bf16 ? run_step<__nv_bfloat16>(c, in, out, m) : run_step<float>(c, in, out, m);
+  if (profile) {
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess && rc == DC_OK)
+      rc = fail(c, DC_ERR_CUDA, "stream sync failed: %s", cudaGetErrorString(e));
+    for (int i = 0; i < DC_STAGE_COUNT; ++i) {
+      stage_ms[i] = 0.f;
+      if (stage_launches) stage_launches[i] = c->prof.launches[i];
+    }
+    if (e == cudaSuccess)
+      for (auto& sp : c->prof.spans) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, sp.a, sp.b);
+        stage_ms[sp.stage] += ms;
+      }
+    c->prof.on = false;
+  }
+  if (dev != c->device && dev >= 0) cudaSetDevice(dev);
+  return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_ctx** out) {
+  if (!cfg || !w || !out) return fail(nullptr, DC_ERR_INVALID_ARG, "null argument");
+  *out = nullptr;
+  const dc_config& g = *cfg;
+  if (g.n_layers < 0 || g.d_model < 1 || g.n_q_heads < 1 || g.n_kv_heads < 1 || g.head_dim < 2 ||
+      g.d_ff < 1 || g.vocab < 2)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "non-positive model dimension");
+  if (g.head_dim % 2) return fail(nullptr, DC_ERR_INVALID_ARG, "head_dim must be even");
+  if (g.n_q_heads % g.n_kv_heads)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
+  if (g.mask_id < 0 || g.mask_id >= g.vocab)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "mask_id outside the vocabulary");
+  if (g.dtype != DC_F32 && g.dtype != DC_BF16) return fail(nullptr, DC_ERR_INVALID_ARG, "dtype");
+  if (g.max_batch < 1 || g.max_batch > DC_MAX_BATCH)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "max_batch outside [1, %d]", DC_MAX_BATCH);
+  if (g.max_window < 16 || g.max_window > DC_MAX_WINDOW || g.max_window % 16)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "max_window must be a multiple of 16 in [16, %d]",
+                DC_MAX_WINDOW);
+  if (g.max_ctx < 0 || g.max_ctx % 64)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "max_ctx must be a non-negative multiple of 64");
+  if (g.max_last < 0) return fail(nullptr, DC_ERR_INVALID_ARG, "max_last negative");
+  if (g.L_min < 1 || g.L_max < 1 || g.smooth_radius < 0 || g.smooth_radius > 8)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "L_min/L_max/smooth_radius out of range");
+  if (g.norm_mode < 0 || g.norm_mode > 2 || g.boundary_mode < 0 || g.boundary_mode > 1 ||
+      g.cap_mode < 0 || g.cap_mode > 1 || g.impl < 0 || g.impl > 1)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "bad mode selector");
+  if (!w->embed || !w->final_norm || !w->lm_head)
+    return fail(nullptr, DC_ERR_INVALID_ARG, "null embed/final_norm/lm_head");
+  if (g.n_layers > 0 && (!w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
+                         !w->w_down || !w->norm1 || !w->norm2))
+    return fail(nullptr, DC_ERR_INVALID_ARG, "null per-layer weight array");
+  for (int l = 0; l < g.n_layers; ++l)
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] ||
+        !w->w_down[l] || !w->norm1[l] || !w->norm2[l])
+      return fail(nullptr, DC_ERR_INVALID_ARG, "null weight pointer in layer %d", l);
+
+  dc_ctx* c = new dc_ctx();
+  c->cfg = g;
+  c->hp = Hyper{g.lambda, g.L_min, g.L_max, g.tau_low, g.tau_high, g.gamma,
+                g.smooth_radius, g.norm_mode, g.boundary_mode, g.cap_mode};
+  c->stream = (cudaStream_t)cuda_stream;
+  if (cudaGetDevice(&c->device) != cudaSuccess) {
+    delete c;
+    cudaGetLastError();
+    return fail(nullptr, DC_ERR_CUDA, "no current CUDA device");
+  }
+  c->bf16 = g.dtype == DC_BF16;
+  c->embed = w->embed; c->final_norm = w->final_norm; c->lm_head = w->lm_head;
+  auto cp = [&](std::vector<const void*>& dst, const void* const* src) {
+    dst.assign(src, src + g.n_layers);
+  };
+  if (g.n_layers > 0) {
+    cp(c->wq, w->wq); cp(c->wk, w->wk); cp(c->wv, w->wv); cp(c->wo, w->wo);
+    cp(c->w_gate, w->w_gate); cp(c->w_up, w->w_up); cp(c->w_down, w->w_down);
+    cp(c->norm1, w->norm1); cp(c->norm2, w->norm2);
+  }
+  c->use_tc = g.impl == DC_IMPL_AUTO && tc_supported(g);
+  const size_t es = c->bf16 ? 2 : 4;
+  c->R_cap_max = round_up(g.max_last + g.max_window, 16);
+  c->M_max = 2 * g.max_batch * c->R_cap_max;
+  const int npos_max = round_up(g.max_batch * g.max_window, 128);
+  c->Mlm_max = 2 * npos_max;
+  const size_t M = c->M_max;
+  const int nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim;
+  bool ok = true;
+  c->x = ws_alloc<float>(c, M * g.d_model, &ok);
+  c->a = ws_alloc<char>(c, M * g.d_model * es, &ok);
+  c->h = ws_alloc<char>(c, (size_t)c->Mlm_max * g.d_model * es, &ok);
+  c->cos_sin = ws_alloc<float>(c, (size_t)g.max_batch * c->R_cap_max * hd, &ok);
+  const size_t nw = (size_t)g.max_batch * g.max_window;
+  c->ws_pred = ws_alloc<int32_t>(c, nw, &ok);
+  c->ws_conf = ws_alloc<float>(c, nw, &ok);
+  c->ws_ent = ws_alloc<float>(c, nw, &ok);
+  c->ws_infl = ws_alloc<float>(c, nw, &ok);
+  c->ws_lse = ws_alloc<float>(c, nw, &ok);
+  if (c->use_tc) {
+    int rc = tc_create(g, c->stream, c->M_max, c->Mlm_max, c->wq, c->wk, c->wv, c->wo, c->w_gate,
+                       c->w_up, c->w_down, c->lm_head, &c->tc);
+    if (rc != DC_OK) {
+      std::string why = c->tc ? tc_error(c->tc) : "tensor-core state allocation failed";
+      dc_destroy(c);
+      return fail(nullptr, rc, "%s", why.c_str());
+    }
+  } else {
+    c->q = ws_alloc<char>(c, M * nq * hd * es, &ok);
+    c->k = ws_alloc<char>(c, M * nkv * hd * es, &ok);
+    c->v = ws_alloc<char>(c, M * nkv * hd * es, &ok);
+    c->o = ws_alloc<char>(c, M * nq * hd * es, &ok);
+    c->act = ws_alloc<char>(c, M * g.d_ff * es, &ok);
+    const size_t tmp_cols = (size_t)((nq + 2 * nkv) * hd > 2 * g.d_ff ? (nq + 2 * nkv) * hd
+                                                                      : 2 * g.d_ff);
+    c->tmp = ws_alloc<float>(c, M * tmp_cols, &ok);
+    c->logits = ws_alloc<float>(c, (size_t)c->Mlm_max * g.vocab, &ok);
+  }
+  if (!ok) {
+    dc_destroy(c);
+    return fail(nullptr, DC_ERR_NOMEM, "workspace allocation failed");
+  }
+  *out = c;
+  return DC_OK;
+}
+
+int dc_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out) {
+  return do_step(c, in, out, false, nullptr, nullptr);
+}
+
+int dc_step_profiled(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, float* stage_ms,
+                     int32_t* stage_launches) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!stage_ms) return fail(c, DC_ERR_INVALID_ARG, "stage_ms null");
+  return do_step(c, in, out, true, stage_ms, stage_launches);
+}
+
+int dc_boundary(dc_ctx* c, const dc_boundary_in* in, const dc_boundary_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !out || !in->influence || !in->entropy || !in->win_len || !out->block_len)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument");
+  SeqMeta m;
+  int rc = build_meta(c, in->batch, 0, nullptr, nullptr, in->win_len, in->remain_len, &m);
+  if (rc != DC_OK) return rc;
+  for (int b = 0; b < m.batch; ++b) m.have_prev[b] = in->have_prev ? (in->have_prev[b] != 0) : 1;
+  launch_boundary(in->influence, in->entropy, c->cfg.max_window, m, c->hp, c->cfg.max_window,
+                  out->score, out->cum_influence, out->cum_score, out->block_len, c->stream);
+  DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
+int dc_select(dc_ctx* c, const dc_select_in* in, const dc_select_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !out || !in->conf || !in->win_ids || !in->xlogp || !in->block_len || !in->win_len)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument");
+  if (!out->sel_mask && !out->sel_idx && !out->sel_count)
+    return fail(c, DC_ERR_INVALID_ARG, "no output requested");
+  SeqMeta m;
+  int rc = build_meta(c, in->batch, 0, nullptr, nullptr, in->win_len, nullptr, &m);
+  if (rc != DC_OK) return rc;
+  Hyper hp = c->hp;
+  if (in->override_thresholds) {
+    hp.tau_low = in->tau_low; hp.tau_high = in->tau_high; hp.gamma = in->gamma;
+  }
+  launch_select(in->conf, in->win_ids, in->xlogp, in->block_len, m, hp, c->cfg.mask_id,
+                c->cfg.max_window, out->sel_mask, out->sel_idx, out->sel_count, c->stream);
+  DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
+int dc_debug_logits(dc_ctx* c, int32_t variant, float* outp) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!outp || variant < 0 || variant > 1) return fail(c, DC_ERR_INVALID_ARG, "bad argument");
+  if (!c->have_logits || !c->logits)
+    return fail(c, DC_ERR_UNSUPPORTED, "logits exist only after a CUDA-core LM head step");
+  const SeqMeta& m = c->last_meta;
+  if (variant >= m.nv) return fail(c, DC_ERR_INVALID_ARG, "the last step ran no prev variant");
+  const int V = c->cfg.vocab;
+  for (int b = 0; b < m.batch; ++b)
+    for (int k = 0; k < m.win_len[b]; ++k) {
+      const float* src = c->logits + (size_t)lm_row(m, variant, b * m.W_cap + k) * V;
+      float* dst = outp + ((size_t)b * c->cfg.max_window + k) * V;
+      if (cudaMemcpyAsync(dst, src, sizeof(float) * V, cudaMemcpyDeviceToDevice, c->stream) !=
+          cudaSuccess)
+        return fail(c, DC_ERR_CUDA, "logit copy failed");
+    }
+  return DC_OK;
+}
+
+int dc_destroy(dc_ctx* c) {
+  if (!c) return DC_OK;
+  if (c->tc) tc_destroy(c->tc);
+  for (void* p : c->allocs) cudaFree(p);
+  delete c;
+  return DC_OK;
+}
+
+const char* dc_last_error(const dc_ctx* c) {
+  return c ? c->err.c_str() : g_create_error.c_str();
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Tensor-core (tcgen05 + TMA) half of the block-step: dense layers, attention, LM head.
+#pragma once
+#include <vector>
+
+#include "kernels.h"
+
+namespace dc {
+
+// Stage bracket used for per-stage timing; a no-op unless profiling.
+struct StageHook {
+  virtual void begin(int stage, int n_launch) = 0;
+  virtual void end() = 0;
+  virtual ~StageHook() {}
+};
+
+struct TcState;
+
+// true if the tensor-core kernels take this model shape
+bool tc_supported(const dc_config& g);
+
+int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
+              const std::vector<const void*>& wq, const std::vector<const void*>& wk,
+              const std::vector<const void*>& wv, const std::vector<const void*>& wo,
+              const std::vector<const void*>& w_gate, const std::vector<const void*>& w_up,
+              const std::vector<const void*>& w_down, const void* lm_head, TcState** out);
+void tc_destroy(TcState* t);
+const char* tc_error(const TcState* t);
+
+// One transformer layer after the first RMSNorm: a = norm1(x) is given; on return the
+// attention and MLP residual updates are applied to x except for the split-K partial sums of
+// the last GEMM, which are handed back (part / nsplit / part_stride) for the next norm to fold.
+int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
+             const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
+             const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
+             StageHook& hook);
+
+// LM head fused with the streaming softmax statistics; fills the workspace signal arrays and
+// the caller's outputs.  Never writes logits.
+int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id, int forbid,
+              int32_t* ws_pred, float* ws_conf, float* ws_ent, float* ws_infl, float* ws_lse,
+              SignalOut out);
+
+}  // namespace dc
