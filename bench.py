@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the DepCap block-step on B200.
+
+One "step" = one whole pass of the hot path over one batch of synthetic input:
+dc_step (embedding, transformer stack over the cached context for the curr and prev variants,
+LM head with the streaming softmax statistics, cross log-probs, block boundary) followed by
+dc_select (CAP-Decoding).  Metric: committed tokens per second = sum_b |S_b| / step time, with
+the block-step latency as ms_per_step.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 runs N independent replicas (one process per GPU, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_15750_b200 import inputs  # noqa: E402
+
+METRIC = "committed_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def _layer_param_count(wl):
+    hq, hkv = wl.n_q_heads * wl.head_dim, wl.n_kv_heads * wl.head_dim
+    return wl.d_model * (hq + 2 * hkv) + hq * wl.d_model + 3 * wl.d_model * wl.d_ff
+
+
+class ClockSampler:
+    def __init__(self, index):
+        self.path = f"/tmp/dc_clocks_{os.getpid()}.csv"
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.f = open(self.path, "w")
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                       "-i", str(index), "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            out = dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=16):
+    """Times the CPU oracle, as it stands, on a bounded sample of the step for sequence 0:
+    one transformer layer (curr and prev variants) and the LM head + signals on the first
+    n_head_pos window positions; the full-step time is extrapolated from the two."""
+    import numpy as np
+    from oracle import adapters
+    from oracle import depcap_oracle as O
+    one = dict(embed=weights_dev["embed"], lm_head=weights_dev["lm_head"],
+               final_norm=weights_dev["final_norm"], layers=weights_dev["layers"][:1])
+    ow = adapters.weights_from_torch(one)
+    ocfg = adapters.config_from_workload(wl, n_layers=1)
+    P, Lb, W = lens["ctx_len"][0], lens["last_len"][0], lens["win_len"][0]
+    kc = adapters.to_np(k_log[:1, 0]) if k_log is not None else None
+    vc = adapters.to_np(v_log[:1, 0]) if v_log is not None else None
+    last = toks["last_ids"][0, :Lb].numpy()
+    win = toks["win_ids"][0, :W].numpy()
+    tok_curr = np.concatenate([last, win]).astype(np.int64)
+    tok_prev = tok_curr.copy(); tok_prev[:Lb] = wl.mask_id
+    t0 = time.perf_counter()
+    O.forward(ocfg, ow, tok_curr, P, kc[:, :, :P] if kc is not None else None,
+              vc[:, :, :P] if vc is not None else None, n_layers=1)
+    O.forward(ocfg, ow, tok_prev, P, kc[:, :, :P] if kc is not None else None,
+              vc[:, :, :P] if vc is not None else None, n_layers=1)
+    t_layer = time.perf_counter() - t0
+    n = min(n_head_pos, W)
+    hf = (adapters.to_np(steer[0, 0, :n]), adapters.to_np(steer[0, 1, :n]))
+    t0 = time.perf_counter()
+    O.step(ocfg, ow, None, None, 0, last, win[:n], lens["remain_len"][0], h_final=hf)
+    t_head = time.perf_counter() - t0
+    est = wl.n_layers * t_layer + t_head * (W / n)
+    return dict(t_layer=t_layer, t_head=t_head, est_step_s=est * wl.batch,
+                sample=f"sequence 0: 1 of {wl.n_layers} layers (curr+prev variants) + LM head/"
+                       f"signals/decisions on {n} of {W} window positions; extrapolated to "
+                       f"{wl.n_layers} layers, {W} positions, batch {wl.batch}")
+
+
+def _oracle_committed(wl, weights_dev, toks, lens, steer):
+    """Committed tokens of the full steered step by the oracle's decisions (not timed): the
+    steering replaces the stack's output, so this needs the LM head only."""
+    from oracle import adapters
+    from oracle import depcap_oracle as O
+    one = dict(embed=weights_dev["embed"][:1], lm_head=weights_dev["lm_head"],
+               final_norm=weights_dev["final_norm"], layers=[])
+    ow = adapters.weights_from_torch(one)
+    ocfg = adapters.config_from_workload(wl, n_layers=0)
+    total = 0
+    for b in range(wl.batch):
+        Lb, W = lens["last_len"][b], lens["win_len"][b]
+        hf = (adapters.to_np(steer[b, 0, :W]), adapters.to_np(steer[b, 1, :W]))
+        o = O.step(ocfg, ow, None, None, 0, toks["last_ids"][b, :Lb].numpy(),
+                   toks["win_ids"][b, :W].numpy(), lens["remain_len"][b], h_final=hf)
+        total += len(o["selected"])
+    return total
+
+
+def _setup(wl, dev, n_layers):
+    weights = inputs.make_weights(wl, device=dev, n_layers=n_layers)
+    k_log, v_log = inputs.make_ctx_kv(wl, device=dev, n_layers=n_layers)
+    toks = inputs.make_tokens(wl)
+    lens = {k: [int(x) for x in v] for k, v in inputs.make_lengths(wl).items()}
+    steer = inputs.make_steering(wl, weights["lm_head"], profile="decay")
+    return weights, k_log, v_log, toks, lens, steer
+
+
+def run_reference(args, wl, rank, world):
+    """The reference arm: the CPU oracle, as it stands, timed on the host cores."""
+    if rank != 0:
+        return
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    n_layers = args.layers or wl.n_layers
+    wl1 = inputs.scaled(wl, n_layers=n_layers)
+    weights = inputs.make_weights(wl, device=dev, n_layers=1)
+    k_log, v_log = inputs.make_ctx_kv(inputs.scaled(wl, n_layers=1), device=dev, n_layers=1)
+    toks = inputs.make_tokens(wl)
+    lens = {k: [int(x) for x in v] for k, v in inputs.make_lengths(wl).items()}
+    steer = inputs.make_steering(wl, weights["lm_head"], profile="decay")
+    committed = _oracle_committed(wl, weights, toks, lens, steer)
+    times = []
+    sample = None
+    for i in range(args.warmup + args.steps):
+        s = _oracle_sample(wl1, weights, k_log, v_log, toks, lens, steer)
+        sample = s["sample"]
+        if i >= args.warmup:
+            times.append(s["est_step_s"])
+    t = sum(times) / len(times)
+    value = committed / t
+    cores = torch.get_num_threads()
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=wl.name, batch=wl.batch, layers=n_layers),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llada8b_b1", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="debug: run fewer layers (invalid as a result)")
+    ap.add_argument("--kernels", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    wl = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl, rank, world)
+        return
+
+    from paper_2604_15750_b200 import DepCap, pack_kv_cache, STAGE_NAMES
+    from paper_2604_15750_b200 import build as _build
+    _build.build()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU path"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    n_layers = args.layers or wl.n_layers
+    # each replica draws its own sequences (seed offset by rank); weights are the same model
+    wl_r = inputs.scaled(wl, seed=wl.seed + 1000 * rank) if rank else wl
+    weights, k_log, v_log, toks, lens, steer = _setup(wl, dev, n_layers)
+    if rank:
+        toks = inputs.make_tokens(wl_r)
+        steer = inputs.make_steering(wl_r, weights["lm_head"], profile="decay")
+    eng = DepCap.from_workload(wl, weights, n_layers=n_layers, impl=1 if args.kernels == "simt" else 0)
+    B, W = wl.batch, eng.max_window
+    kc, vc = pack_kv_cache(k_log, v_log, eng.max_batch, eng.max_ctx)
+    last_h = torch.zeros((B, eng.max_last), dtype=torch.int32).pin_memory()
+    last_h[:, :wl.last_len] = toks["last_ids"]
+    win_h = torch.full((B, W), wl.mask_id, dtype=torch.int32).pin_memory()
+    win_h[:, :wl.win_len] = toks["win_ids"]
+    hf_h = torch.zeros((B, 2, W, wl.d_model), dtype=wl.torch_dtype).pin_memory()
+    hf_h[:, :, :wl.win_len] = steer.cpu()
+    last_d, win_d, hf_d = last_h.to(dev), win_h.to(dev), hf_h.to(dev)
+    step_kw = dict(k_cache=kc, v_cache=vc, ctx_len=lens["ctx_len"], last_len=lens["last_len"],
+                   win_len=lens["win_len"], remain_len=lens["remain_len"])
+    stream = eng.stream
+
+    def one_step():
+        eng.step(last_ids=last_d, win_ids=win_d, h_final=hf_d, **step_kw)
+        eng.select(win_d, lens["win_len"])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    committed = int(eng.sel["sel_count"][:B].sum().item())
+    status_bad = int(eng.out["status"][:B].abs().max().item())
+
+    # ---- end to end through the public API with host buffers ------------------------------
+    out_h = dict(pred=torch.zeros((B, W), dtype=torch.int32).pin_memory(),
+                 conf=torch.zeros((B, W), dtype=torch.float32).pin_memory(),
+                 blk=torch.zeros((B,), dtype=torch.int32).pin_memory(),
+                 mask=torch.zeros((B, W), dtype=torch.uint8).pin_memory(),
+                 cnt=torch.zeros((B,), dtype=torch.int32).pin_memory())
+
+    def one_step_e2e():
+        with torch.cuda.stream(stream):
+            last_d.copy_(last_h, non_blocking=True)
+            win_d.copy_(win_h, non_blocking=True)
+            hf_d.copy_(hf_h, non_blocking=True)
+            one_step()
+            out_h["pred"].copy_(eng.out["pred_id"][:B], non_blocking=True)
+            out_h["conf"].copy_(eng.out["conf"][:B], non_blocking=True)
+            out_h["blk"].copy_(eng.out["block_len"][:B], non_blocking=True)
+            out_h["mask"].copy_(eng.sel["sel_mask"][:B], non_blocking=True)
+            out_h["cnt"].copy_(eng.sel["sel_count"][:B], non_blocking=True)
+        stream.synchronize()          # the host needs the subset before it can commit tokens
+
+    h2d = last_h.numel() * 4 + win_h.numel() * 4 + hf_h.numel() * hf_h.element_size()
+    d2h = sum(t.numel() * t.element_size() for t in out_h.values())
+    e2e_steps = max(3, min(args.steps, 10))
+    one_step_e2e()
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    for _ in range(e2e_steps):
+        one_step_e2e()
+    e3.record(stream)
+    barrier()
+    e2e_ms = e2.elapsed_time(e3) / e2e_steps
+    committed_e2e = int(out_h["cnt"].sum().item())
+
+    # ---- per-stage device time, live, for the roofline of the dominant kernel --------------
+    stage_ms = {n: 0.0 for n in STAGE_NAMES}
+    launches = {}
+    reps = 3
+    for _ in range(reps):
+        ms, launches = eng.step_profiled(last_ids=last_d, win_ids=win_d, h_final=hf_d, **step_kw)
+        for n in STAGE_NAMES:
+            stage_ms[n] += ms[n] / reps
+    gpu_launches = (sum(launches.values()) + 1) * args.steps      # + dc_select
+
+    # ---- reduce over ranks --------------------------------------------------------------------
+    ms_step = ms_total / args.steps
+    if dist is not None:
+        t = torch.tensor([ms_step, e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, e2e_ms = float(t[0]), float(t[1])
+        cnt = torch.tensor([committed, committed_e2e], device=dev, dtype=torch.int64)
+        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
+        committed, committed_e2e = int(cnt[0]), int(cnt[1])
+    if rank != 0:
+        eng.close()
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    gemm_ms = sum(stage_ms[n] for n in ("qkv", "oproj", "gateup", "down"))
+    M = 2 * wl.batch * ((wl.last_len + wl.win_len + 15) // 16 * 16)
+    w_bytes = 2.0 * _layer_param_count(wl) * n_layers
+    flops = 2.0 * _layer_param_count(wl) * n_layers * M
+    t_hbm = w_bytes / (peaks["hbm"] * 1e9)
+    t_tensor = flops / (peaks["bf16_sustained"] * 1e12)
+    if t_hbm >= t_tensor:
+        ach = w_bytes / (gemm_ms * 1e-3) / 1e9
+        roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm"], unit="GB/s",
+                    frac=ach / peaks["hbm"])
+    else:
+        ach = flops / (gemm_ms * 1e-3) / 1e12
+        roof = dict(bound="tensor", achieved=ach, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                    frac=ach / peaks["bf16_sustained"])
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dense_gemm_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            tj = json.load(open(tpath))
+            traffic = tj["dram_bytes_per_layer"] * n_layers if wl.name == tj.get("workload") else None
+        except Exception:
+            traffic = None
+    roof.update(kernel="dense-layer GEMMs (QKV, O, gate/up, down), all layers of one step",
+                traffic=traffic, peak_source=peaks["source"] + " (of measured)" if peaks["source"] == "measured"
+                else "fallback (of fallback)", stage_ms={k: round(v, 4) for k, v in stage_ms.items()})
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        s = _oracle_sample(inputs.scaled(wl, n_layers=n_layers), weights,
+                           k_log, v_log, toks, lens, steer)
+        oc = _oracle_committed(wl, weights, toks, lens, steer)
+        cpu = dict(value=oc / s["est_step_s"], unit=UNIT, cores=torch.get_num_threads(),
+                   kind="oracle", sample=s["sample"], est_step_ms=s["est_step_s"] * 1e3,
+                   committed=oc)
+
+    line = dict(metric=METRIC, value=committed / (ms_step * 1e-3), unit=UNIT, n_gpus=world,
+                steps=args.steps, warmup=args.warmup, ms_per_step=ms_step, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="bf16" if wl.dtype == "bf16" else "f32",
+                data="synthetic",
+                config=dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
+                            window=wl.win_len, layers=n_layers, variants="curr+prev",
+                            steering="decay", committed_per_step=committed,
+                            l2="inputs larger than L2 (weights streamed every step)",
+                            kernels=args.kernels, status=status_bad),
+                clocks=clocks,
+                e2e=dict(value=committed_e2e / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
+                         h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
+                gpu_launches=gpu_launches, roofline=roof, cpu_baseline=cpu)
+    print(json.dumps(line))
+    eng.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -236,7 +236,7 @@ class DepCap:
 
     # -- dc_step ---------------------------------------------------------------------------
     def _step_structs(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len,
-                      remain_len, influence, boundary, h_final, want_xlogp=True):
+                      remain_len, influence=True, boundary=True, h_final=None, want_xlogp=True):
         B = len(win_len)
         self._keep = (k_cache, v_cache, last_ids, win_ids, h_final,
                       _host_i32(ctx_len, B), _host_i32(last_len, B), _host_i32(win_len, B),

@@ -104,7 +104,7 @@ def test_argument_errors_are_reported_on_the_host_and_leave_outputs_untouched():
     eng = case.make_engine()
     di = case.device_inputs(eng)
     eng.out["pred_id"].fill_(-7)
-    bad = dict(di); bad["win_len"] = [25, 24, 24]           # > max_window (24)
+    bad = dict(di); bad["win_len"] = [33, 24, 24]           # > max_window (32)
     with pytest.raises(DepCapError) as e:
         eng.step(**bad)
     assert e.value.code == 2 and "win_len" in str(e.value)
