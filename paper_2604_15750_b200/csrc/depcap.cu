@@ -61,7 +61,8 @@ struct dc_ctx {
   cudaStream_t stream = nullptr;
   int device = 0;
   bool bf16 = false;
-  bool use_tc = false;  // tensor-core kernels for the dense layers / LM head / attention
+  bool use_tc = false;  // tensor-core kernels for the transformer layers
+  bool tc_lm = false;   // tensor-core LM head fused with the streaming softmax statistics
   const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
   std::vector<const void*> wq, wk, wv, wo, w_gate, w_up, w_down, norm1, norm2;
   // capacities
@@ -230,7 +231,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
   pf.end();
 
   SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, g.max_window};
-  if (c->use_tc) {
+  if (c->tc_lm) {
     pf.begin(DC_STAGE_LMHEAD, 2);
     int rc = tc_lmhead(c->tc, m, (const __nv_bfloat16*)h, g.mask_id, g.forbid_mask_pred,
                        c->ws_pred, c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so);
@@ -258,6 +259,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
                     out->cum_influence, out->cum_score, out->block_len, s);
     pf.end();
   }
+  if (c->use_tc) tc_flush_status(c->tc, out->status, m.batch);
   DC_CHECK_LAUNCH(c);
   c->last_meta = m;
   return DC_OK;
@@ -375,6 +377,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
     cp(c->norm1, w->norm1); cp(c->norm2, w->norm2);
   }
   c->use_tc = g.impl == DC_IMPL_AUTO && tc_supported(g);
+  c->tc_lm = c->use_tc && tc_has_lmhead(g);
   const size_t es = c->bf16 ? 2 : 4;
   c->R_cap_max = round_up(g.max_last + g.max_window, 16);
   c->M_max = 2 * g.max_batch * c->R_cap_max;
@@ -410,8 +413,8 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
     const size_t tmp_cols = (size_t)((nq + 2 * nkv) * hd > 2 * g.d_ff ? (nq + 2 * nkv) * hd
                                                                       : 2 * g.d_ff);
     c->tmp = ws_alloc<float>(c, M * tmp_cols, &ok);
-    c->logits = ws_alloc<float>(c, (size_t)c->Mlm_max * g.vocab, &ok);
   }
+  if (!c->tc_lm) c->logits = ws_alloc<float>(c, (size_t)c->Mlm_max * g.vocab, &ok);
   if (!ok) {
     dc_destroy(c);
     return fail(nullptr, DC_ERR_NOMEM, "workspace allocation failed");

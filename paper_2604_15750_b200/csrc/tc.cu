@@ -1,21 +1,290 @@
+// Host side of the tensor-core path: tensor maps, workspace, launch configuration.
 #include "tc.h"
+
+#include <cuda.h>
+#include <stdarg.h>
+#include <stdio.h>
+
+#include <map>
+#include <string>
+
+#include "tc_gemm.cuh"
 
 namespace dc {
 
-struct TcState { const char* err = ""; };
+namespace {
 
-bool tc_supported(const dc_config&) { return false; }
-int tc_create(const dc_config&, cudaStream_t, int, int, const std::vector<const void*>&,
-              const std::vector<const void*>&, const std::vector<const void*>&,
-              const std::vector<const void*>&, const std::vector<const void*>&,
-              const std::vector<const void*>&, const std::vector<const void*>&, const void*,
-              TcState** out) { *out = nullptr; return DC_ERR_UNSUPPORTED; }
-void tc_destroy(TcState* t) { delete t; }
-const char* tc_error(const TcState* t) { return t ? t->err : ""; }
-int tc_layer(TcState*, int, const SeqMeta&, float*, const __nv_bfloat16*, const __nv_bfloat16*,
-             const __nv_bfloat16*, const float*, const __nv_bfloat16*, const float**, int*,
-             size_t*, StageHook&) { return DC_ERR_UNSUPPORTED; }
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
+            cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns (128 bytes) x box_rows rows,
+// 128-byte swizzle, zero fill outside the tensor
+bool make_map_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kSmemBudget = 232448 - 1024;  // opt-in shared memory per CTA, minus alignment slack
+constexpr int kStaticQkv = 128 * 33 * 4 + 512;  // static shared memory of the kernels (upper bounds)
+constexpr int kStaticOther = 512;
+
+}  // namespace
+
+struct LayerMaps {
+  CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down;
+};
+
+struct ActMaps {
+  CUtensorMap a, o, act;
+};
+
+struct TcState {
+  dc_config g{};
+  cudaStream_t s = nullptr;
+  int M_max = 0;
+  std::vector<LayerMaps> layers;
+  std::map<int, ActMaps> act_maps;  // keyed by BN
+  std::vector<void*> allocs;
+  __nv_bfloat16 *a_buf = nullptr;  // borrowed: the normed activations of the scheduler
+  __nv_bfloat16 *q = nullptr, *k = nullptr, *v = nullptr, *o = nullptr, *act = nullptr;
+  float* part = nullptr;
+  size_t part_stride = 0;
+  int max_split = 4;
+  int32_t* status = nullptr;
+  std::string err;
+  bool attrs_set = false;
+};
+
+namespace {
+
+int tfail(TcState* t, int code, const char* fmt, ...) {
+  char buf[400];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  t->err = buf;
+  return code;
+}
+
+template <typename T>
+T* talloc(TcState* t, size_t n, bool* ok) {
+  void* p = nullptr;
+  if (cudaMalloc(&p, (n ? n : 1) * sizeof(T)) != cudaSuccess) {
+    cudaGetLastError();
+    *ok = false;
+    return nullptr;
+  }
+  t->allocs.push_back(p);
+  return reinterpret_cast<T*>(p);
+}
+
+int pick_bn(int M) {
+  const int nblk = (M + 255) / 256;
+  const int bn = ((M + nblk - 1) / nblk + 15) / 16 * 16;
+  return bn;
+}
+
+}  // namespace
+
+bool tc_supported(const dc_config& g) {
+  return g.dtype == DC_BF16 && g.head_dim == 128 && g.d_model % 128 == 0 && g.d_ff % 128 == 0 &&
+         g.n_layers > 0 && get_encode() != nullptr;
+}
+
+const char* tc_error(const TcState* t) { return t ? t->err.c_str() : ""; }
+
+void tc_destroy(TcState* t) {
+  if (!t) return;
+  for (void* p : t->allocs) cudaFree(p);
+  delete t;
+}
+
+int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
+              const std::vector<const void*>& wq, const std::vector<const void*>& wk,
+              const std::vector<const void*>& wv, const std::vector<const void*>& wo,
+              const std::vector<const void*>& w_gate, const std::vector<const void*>& w_up,
+              const std::vector<const void*>& w_down, const void* lm_head, TcState** out) {
+  (void)Mlm_max; (void)lm_head;
+  TcState* t = new TcState();
+  *out = t;
+  t->g = g; t->s = s; t->M_max = M_max;
+  const uint64_t d = g.d_model, hq = (uint64_t)g.n_q_heads * g.head_dim,
+                 hkv = (uint64_t)g.n_kv_heads * g.head_dim, F = g.d_ff;
+  t->layers.resize(g.n_layers);
+  for (int l = 0; l < g.n_layers; ++l) {
+    LayerMaps& L = t->layers[l];
+    bool ok = make_map_2d(&L.wq, wq[l], hq, d, 128) && make_map_2d(&L.wk, wk[l], hkv, d, 128) &&
+              make_map_2d(&L.wv, wv[l], hkv, d, 128) && make_map_2d(&L.wo, wo[l], d, hq, 128) &&
+              make_map_2d(&L.w_gate, w_gate[l], F, d, 128) &&
+              make_map_2d(&L.w_up, w_up[l], F, d, 128) && make_map_2d(&L.w_down, w_down[l], d, F, 128);
+    if (!ok) return tfail(t, DC_ERR_CUDA, "tensor map encoding failed for layer %d (weights must be 16-byte aligned)", l);
+  }
+  bool ok = true;
+  const size_t M = M_max;
+  t->q = talloc<__nv_bfloat16>(t, M * hq, &ok);
+  t->k = talloc<__nv_bfloat16>(t, M * hkv, &ok);
+  t->v = talloc<__nv_bfloat16>(t, M * hkv, &ok);
+  t->o = talloc<__nv_bfloat16>(t, M * hq, &ok);
+  t->act = talloc<__nv_bfloat16>(t, M * F, &ok);
+  t->part_stride = M * d;
+  t->part = talloc<float>(t, (size_t)t->max_split * t->part_stride, &ok);
+  t->status = talloc<int32_t>(t, 4, &ok);
+  if (!ok) return tfail(t, DC_ERR_NOMEM, "tensor-core workspace allocation failed");
+  cudaMemsetAsync(t->status, 0, 4 * sizeof(int32_t), s);
+  cudaError_t e1 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_QKV>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kSmemBudget + 1024 - kStaticQkv);
+  cudaError_t e2 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_PARTIAL>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kSmemBudget + 1024 - kStaticOther);
+  cudaError_t e3 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_SWIGLU>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kSmemBudget + 1024 - kStaticOther);
+  if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+    cudaGetLastError();
+    return tfail(t, DC_ERR_CUDA, "cannot opt in to %d bytes of shared memory", kSmemBudget);
+  }
+  return DC_OK;
+}
+
+static int get_act_maps(TcState* t, const __nv_bfloat16* a, int BN, ActMaps** out) {
+  auto it = t->act_maps.find(BN);
+  if (it == t->act_maps.end() || t->a_buf != a) {
+    const dc_config& g = t->g;
+    ActMaps am;
+    const uint64_t hq = (uint64_t)g.n_q_heads * g.head_dim;
+    bool ok = make_map_2d(&am.a, a, t->M_max, g.d_model, BN) &&
+              make_map_2d(&am.o, t->o, t->M_max, hq, BN) &&
+              make_map_2d(&am.act, t->act, t->M_max, g.d_ff, BN);
+    if (!ok) return tfail(t, DC_ERR_CUDA, "activation tensor map encoding failed");
+    if (t->a_buf != a) t->act_maps.clear();
+    t->a_buf = const_cast<__nv_bfloat16*>(a);
+    it = t->act_maps.insert_or_assign(BN, am).first;
+  }
+  *out = &it->second;
+  return DC_OK;
+}
+
+template <int EPI>
+static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
+                       const CUtensorMap& w2, const CUtensorMap& ma, GemmParams p, int tiles,
+                       int static_smem) {
+  const int nw = (EPI == GEMM_EPI_SWIGLU) ? 2 : 1;
+  const int sb = gemm_stage_bytes(nw, p.BN);
+  int stages = (kSmemBudget - static_smem) / sb;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return tfail(t, DC_ERR_UNSUPPORTED, "activation block too large for the smem ring");
+  const size_t smem = (size_t)stages * sb + 1024;
+  dim3 grid(tiles, p.nsplit, (p.M + p.BN - 1) / p.BN);
+  p.status = t->status;
+  k_gemm_tc<EPI><<<grid, kGemmThreads, smem, t->s>>>(w0, w1, w2, ma, p, stages);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "GEMM launch failed: %s", cudaGetErrorString(e));
+  return DC_OK;
+}
+
+static int pick_split(int tiles, int KB, int max_split) {
+  // enough CTAs to cover the SMs, at least 8 k-blocks each
+  int s = 148 / tiles;
+  if (s < 1) s = 1;
+  if (s > max_split) s = max_split;
+  while (s > 1 && KB / s < 8) --s;
+  return s;
+}
+
+int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
+             const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
+             const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
+             StageHook& hook) {
+  const dc_config& g = t->g;
+  const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
+  const int M = m.nv * m.batch * m.R_cap;
+  const int BN = pick_bn(M);
+  ActMaps* am = nullptr;
+  int rc = get_act_maps(t, a, BN, &am);
+  if (rc != DC_OK) return rc;
+  const LayerMaps& L = t->layers[layer];
+  GemmParams p{};
+  p.M = M; p.BN = BN; p.nq = nq; p.nkv = nkv; p.hd = hd;
+  p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
+  p.q = t->q; p.k = t->k; p.v = t->v; p.act = t->act;
+  p.part = t->part; p.part_stride = t->part_stride;
+
+  hook.begin(DC_STAGE_QKV, 1);
+  p.N = (nq + 2 * nkv) * hd; p.K = d; p.nsplit = 1;
+  rc = launch_gemm<GEMM_EPI_QKV>(t, L.wq, L.wk, L.wv, am->a, p, nq + 2 * nkv, kStaticQkv);
+  hook.end();
+  if (rc != DC_OK) return rc;
+
+  hook.begin(DC_STAGE_ATTN, 1);
+  launch_attn_simt<__nv_bfloat16>(t->q, t->k, t->v, k_cache, v_cache, g.max_ctx, m, nq, nkv, hd,
+                                  t->o, t->s);
+  hook.end();
+
+  hook.begin(DC_STAGE_OPROJ, 1);
+  p.N = d; p.K = nq * hd; p.nsplit = pick_split(d / kTileN, p.K / kTileK, t->max_split);
+  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.wo, L.wo, L.wo, am->o, p, d / kTileN, kStaticOther);
+  hook.end();
+  if (rc != DC_OK) return rc;
+
+  hook.begin(DC_STAGE_NORM, 1);
+  launch_rmsnorm<__nv_bfloat16>(x, t->part, p.nsplit, t->part_stride, norm2, g.rms_eps, M, d,
+                                const_cast<__nv_bfloat16*>(a), t->s);
+  hook.end();
+
+  hook.begin(DC_STAGE_GATEUP, 1);
+  p.N = F; p.K = d; p.nsplit = 1;
+  rc = launch_gemm<GEMM_EPI_SWIGLU>(t, L.w_gate, L.w_up, L.w_up, am->a, p, F / kTileN, kStaticOther);
+  hook.end();
+  if (rc != DC_OK) return rc;
+
+  hook.begin(DC_STAGE_DOWN, 1);
+  p.N = d; p.K = F; p.nsplit = pick_split(d / kTileN, p.K / kTileK, t->max_split);
+  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.w_down, L.w_down, L.w_down, am->act, p, d / kTileN, kStaticOther);
+  hook.end();
+  if (rc != DC_OK) return rc;
+
+  *part = t->part; *nsplit = p.nsplit; *part_stride = t->part_stride;
+  return DC_OK;
+}
+
 int tc_lmhead(TcState*, const SeqMeta&, const __nv_bfloat16*, int, int, int32_t*, float*, float*,
               float*, float*, SignalOut) { return DC_ERR_UNSUPPORTED; }
+
+bool tc_has_lmhead(const dc_config&) { return false; }
+
+__global__ void k_flush_status(int32_t* tc_status, int32_t* status, int batch) {
+  if (*tc_status != 0) {
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) status[b] = *tc_status;
+    __syncthreads();
+    if (threadIdx.x == 0) *tc_status = 0;
+  }
+}
+
+void tc_flush_status(TcState* t, int32_t* status, int batch) {
+  k_flush_status<<<1, 32, 0, t->s>>>(t->status, status, batch);
+}
 
 }  // namespace dc

@@ -17,6 +17,10 @@ struct TcState;
 
 // true if the tensor-core kernels take this model shape
 bool tc_supported(const dc_config& g);
+// true if the fused tensor-core LM head takes this model shape
+bool tc_has_lmhead(const dc_config& g);
+// copies a device-side timeout raised by a tensor-core kernel into status[0..batch) and clears it
+void tc_flush_status(TcState* t, int32_t* status, int batch);
 
 int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
               const std::vector<const void*>& wq, const std::vector<const void*>& wk,

@@ -1,0 +1,242 @@
+// Weight-streaming bf16 GEMM on tcgen05 for the dense layers of the block-step.
+//
+// out[m, n] = sum_k A[m, k] * W[n, k]        A: activations [M, K], W: weights [N, K]
+//
+// The step has few activation rows (M = 2 * batch * rows, 192 for one sequence) and very many
+// weight rows, so the roles of the MMA operands are swapped: a CTA owns 128 weight rows (the MMA
+// "M" side, one TMEM lane per output feature) and a block of up to 256 activation rows (the MMA
+// "N" side, one TMEM column per row).  Every weight byte is read from HBM exactly once per
+// column block; the activation tile is re-read from L2.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = epilogue (TMEM -> registers -> global).  Shared memory is a ring of kStages
+// slots, each {NW weight tiles 128 x 64, one activation tile BN x 64}, all in the 128-byte
+// swizzled K-major layout that both TMA and tcgen05.mma understand.
+#pragma once
+#include "kernels.h"
+#include "tc_ptx.cuh"
+
+namespace dc {
+
+enum GemmEpi {
+  GEMM_EPI_QKV = 0,      // rotate q/k heads (RoPE), round to bf16, store q, k, v
+  GEMM_EPI_PARTIAL = 1,  // fp32 split-K partial sums [split][M][N]
+  GEMM_EPI_SWIGLU = 2    // two accumulators (gate, up): bf16 silu(gate) * up
+};
+
+struct GemmParams {
+  int M;          // valid activation rows
+  int N;          // weight rows of one matrix (output features)
+  int K;          // reduction length
+  int BN;         // activation rows per column block (multiple of 16, <= 256)
+  int nsplit;     // split-K factor
+  // QKV epilogue
+  int nq, nkv, hd;          // tiles [0,nq) are q heads, [nq,nq+nkv) k heads, rest v heads
+  const float* cos_sin;     // RoPE table [(b, r)][hd]
+  int rows_per_variant;     // batch * R_cap: the table is shared by the variants
+  __nv_bfloat16 *q, *k, *v; // outputs [M, nq*hd], [M, nkv*hd], [M, nkv*hd]
+  // PARTIAL epilogue
+  float* part;              // [nsplit][M_ld][N]
+  size_t part_stride;       // elements between splits
+  // SWIGLU epilogue
+  __nv_bfloat16* act;       // [M, N]
+  int32_t* status;          // device status word(s); DC_ERR_TIMEOUT on an expired wait
+};
+
+constexpr int kGemmThreads = 192;
+constexpr int kTileN = 128;  // weight rows per CTA tile
+constexpr int kTileK = 64;   // bf16 elements per k-block (one 128-byte swizzle row)
+
+__host__ __device__ inline int gemm_stage_bytes(int nw, int BN) {
+  return nw * kTileN * kTileK * 2 + BN * kTileK * 2;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
+          const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a,
+          const GemmParams p, const int stages) {
+  constexpr int NW = (EPI == GEMM_EPI_SWIGLU) ? 2 : 1;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+  __shared__ float xch[(EPI == GEMM_EPI_QKV) ? 128 * 33 : 1];
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x;   // weight tile
+  const int split = blockIdx.y;  // K split
+  const int cblk = blockIdx.z;   // activation column block
+  const int stage_bytes = gemm_stage_bytes(NW, p.BN);
+  const int KB = p.K / kTileK;
+  const int kb0 = (int)(((long long)split * KB) / p.nsplit);
+  const int kb1 = (int)(((long long)(split + 1) * KB) / p.nsplit);
+  const int nkb = kb1 - kb0;
+  const uint32_t tmem_cols = (NW == 2) ? 512u : 256u;
+
+  // which weight matrix and which row of it this tile starts at
+  const CUtensorMap* map_w = &map_w0;
+  int wrow = tile * kTileN;
+  if (EPI == GEMM_EPI_QKV) {
+    if (tile >= p.nq + p.nkv) { map_w = &map_w2; wrow = (tile - p.nq - p.nkv) * kTileN; }
+    else if (tile >= p.nq) { map_w = &map_w1; wrow = (tile - p.nq) * kTileN; }
+  }
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < stages; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
+    ptx::mbar_init(&bar_acc, 1);
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(map_w);
+    ptx::prefetch_tmap(&map_a);
+    if (NW == 2) ptx::prefetch_tmap(&map_w1);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&tmem_base_s, tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (ptx::elect_one()) {
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = (uint32_t)(i / stages) & 1u;
+        if (!ptx::mbar_wait(&bar_empty[s], ph ^ 1u, &abort_flag)) break;
+        uint8_t* slot = smem + (size_t)s * stage_bytes;
+        ptx::mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
+        const int kc = (kb0 + i) * kTileK;
+        ptx::tma_load_2d(slot, map_w, &bar_full[s], kc, wrow);
+        if (NW == 2) ptx::tma_load_2d(slot + kTileN * kTileK * 2, &map_w1, &bar_full[s], kc, wrow);
+        ptx::tma_load_2d(slot + NW * kTileN * kTileK * 2, &map_a, &bar_full[s], kc, cblk * p.BN);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (ptx::elect_one()) {
+      const uint32_t idesc = ptx::idesc_bf16(kTileN, p.BN);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = (uint32_t)(i / stages) & 1u;
+        ok = ptx::mbar_wait(&bar_full[s], ph, &abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t slot = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t dw0 = ptx::smem_desc_sw128(slot);
+        const uint64_t dw1 = ptx::smem_desc_sw128(slot + kTileN * kTileK * 2);
+        const uint64_t da = ptx::smem_desc_sw128(slot + NW * kTileN * kTileK * 2);
+#pragma unroll
+        for (int kk = 0; kk < kTileK / 16; ++kk) {
+          const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
+          // +32 bytes per 16 bf16 along K = +2 in the 16-byte units of the start address
+          ptx::umma_bf16(tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
+          if (NW == 2) ptx::umma_bf16(tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc, acc);
+        }
+        ptx::umma_commit(&bar_empty[s]);  // slot free once these MMAs have read it
+      }
+      ptx::umma_commit(&bar_acc);         // accumulators complete
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+    const int quarter = warp & 3;
+    const int f = quarter * 32 + lane;  // feature (weight row) inside the tile = TMEM lane
+    const bool ok = ptx::mbar_wait(&bar_acc, 0, &abort_flag);
+    ptx::tc_fence_after();
+    if (ok && nkb > 0) {
+      const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const int m_base = cblk * p.BN;
+      for (int c0 = 0; c0 < p.BN; c0 += 32) {
+        float acc[32];
+        // BN is a multiple of 16: the last chunk may be 16 wide
+        const int width = (p.BN - c0 >= 32) ? 32 : 16;
+        if (width == 32) ptx::tmem_ld_32x32(t_lane + c0, acc);
+        else {
+          float a16[16];
+          ptx::tmem_ld_32x16(t_lane + c0, a16);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { acc[j] = a16[j]; acc[16 + j] = 0.f; }
+        }
+        ptx::tmem_ld_wait();
+        if (EPI == GEMM_EPI_PARTIAL) {
+          float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kTileN + f);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int m = m_base + c0 + j;
+            if (j < width && m < p.M) dst[(size_t)m * p.N] = acc[j];
+          }
+        } else if (EPI == GEMM_EPI_SWIGLU) {
+          float up[32];
+          if (width == 32) ptx::tmem_ld_32x32(t_lane + 256 + c0, up);
+          else {
+            float a16[16];
+            ptx::tmem_ld_32x16(t_lane + 256 + c0, a16);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { up[j] = a16[j]; up[16 + j] = 0.f; }
+          }
+          ptx::tmem_ld_wait();
+          __nv_bfloat16* dst = p.act + (size_t)(tile * kTileN + f);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int m = m_base + c0 + j;
+            if (j < width && m < p.M) {
+              const float g = acc[j];
+              dst[(size_t)m * p.N] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * up[j]);
+            }
+          }
+        } else {  // GEMM_EPI_QKV
+          const bool is_v = tile >= p.nq + p.nkv;
+          if (is_v) {
+            __nv_bfloat16* dst = p.v + (size_t)((tile - p.nq - p.nkv) * p.hd + f);
+            const int ld = p.nkv * p.hd;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int m = m_base + c0 + j;
+              if (j < width && m < p.M) dst[(size_t)m * ld] = __float2bfloat16_rn(acc[j]);
+            }
+          } else {
+            // rotate-half RoPE: feature i < hd/2 pairs with i + hd/2, held by the warp two
+            // quarters away; exchange the chunk through shared memory
+#pragma unroll
+            for (int j = 0; j < 32; ++j) xch[f * 33 + j] = acc[j];
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int half = p.hd / 2;
+            const int i = f % half;
+            const bool lo = f < half;
+            const bool is_k = tile >= p.nq;
+            __nv_bfloat16* dst = is_k ? p.k + (size_t)((tile - p.nq) * p.hd + f)
+                                      : p.q + (size_t)(tile * p.hd + f);
+            const int ld = is_k ? p.nkv * p.hd : p.nq * p.hd;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int m = m_base + c0 + j;
+              if (j < width && m < p.M) {
+                const float other = xch[(f ^ half) * 33 + j];
+                const float* cs = p.cos_sin + (size_t)(m % p.rows_per_variant) * p.hd;
+                const float c = cs[i], sn = cs[half + i];
+                const float y = lo ? (acc[j] * c - other * sn) : (acc[j] * c + other * sn);
+                dst[(size_t)m * ld] = __float2bfloat16_rn(y);
+              }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+          }
+        }
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, tmem_cols);
+  }
+  if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, DC_ERR_TIMEOUT);
+}
+
+}  // namespace dc
