@@ -190,8 +190,9 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     const T* kc = in->k_cache ? (const T*)in->k_cache + (size_t)l * k_layer : nullptr;
     const T* vc = in->v_cache ? (const T*)in->v_cache + (size_t)l * k_layer : nullptr;
     if (c->use_tc) {
-      int rc = tc_layer(c->tc, l, m, c->x, (const __nv_bfloat16*)a, (const __nv_bfloat16*)kc,
-                        (const __nv_bfloat16*)vc, c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
+      int rc = tc_layer(c->tc, l, m, c->x, (const __nv_bfloat16*)a,
+                        (const __nv_bfloat16*)in->k_cache, (const __nv_bfloat16*)in->v_cache,
+                        c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
                         &part, &nsplit, &part_stride, pf);
       if (rc != DC_OK) return fail(c, rc, "tensor-core layer %d failed: %s", l, tc_error(c->tc));
       continue;

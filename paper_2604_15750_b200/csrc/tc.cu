@@ -8,6 +8,7 @@
 #include <map>
 #include <string>
 
+#include "tc_attn.cuh"
 #include "tc_gemm.cuh"
 
 namespace dc {
@@ -45,6 +46,20 @@ bool make_map_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D bf16 tensor [n2][n1][n0] (n0 contiguous), box = 64 x box1 x 1, 128-byte swizzle
+bool make_map_3d(CUtensorMap* m, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
+                 uint32_t box1) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[3] = {n0, n1, n2};
+  cuuint64_t strides[2] = {n0 * 2, n0 * n1 * 2};
+  cuuint32_t box[3] = {64, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr int kSmemBudget = 232448 - 1024;  // opt-in shared memory per CTA, minus alignment slack
 constexpr int kStaticQkv = 128 * 33 * 4 + 512;  // static shared memory of the kernels (upper bounds)
 constexpr int kStaticOther = 512;
@@ -72,6 +87,9 @@ struct TcState {
   size_t part_stride = 0;
   int max_split = 4;
   int32_t* status = nullptr;
+  int ldv = 0;  // row pitch of the transposed active V
+  CUtensorMap map_q, map_k, map_vt, map_kc, map_vc;
+  const void *kc_base = nullptr, *vc_base = nullptr;
   std::string err;
   bool attrs_set = false;
 };
@@ -145,7 +163,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
   const size_t M = M_max;
   t->q = talloc<__nv_bfloat16>(t, M * hq, &ok);
   t->k = talloc<__nv_bfloat16>(t, M * hkv, &ok);
-  t->v = talloc<__nv_bfloat16>(t, M * hkv, &ok);
+  t->ldv = (M_max + 63) / 64 * 64;
+  t->v = talloc<__nv_bfloat16>(t, (size_t)t->ldv * hkv, &ok);
   t->o = talloc<__nv_bfloat16>(t, M * hq, &ok);
   t->act = talloc<__nv_bfloat16>(t, M * F, &ok);
   t->part_stride = M * d;
@@ -153,6 +172,20 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
   t->status = talloc<int32_t>(t, 4, &ok);
   if (!ok) return tfail(t, DC_ERR_NOMEM, "tensor-core workspace allocation failed");
   cudaMemsetAsync(t->status, 0, 4 * sizeof(int32_t), s);
+  // active rows beyond the step's M are read by the attention tiles (and masked): keep them finite
+  cudaMemsetAsync(t->q, 0, M * hq * 2, s);
+  cudaMemsetAsync(t->k, 0, M * hkv * 2, s);
+  cudaMemsetAsync(t->v, 0, (size_t)t->ldv * hkv * 2, s);
+  cudaMemsetAsync(t->o, 0, M * hq * 2, s);
+  if (!(make_map_2d(&t->map_q, t->q, M, hq, 128) && make_map_2d(&t->map_k, t->k, M, hkv, 128) &&
+        make_map_2d(&t->map_vt, t->v, hkv, t->ldv, 128)))
+    return tfail(t, DC_ERR_CUDA, "attention tensor map encoding failed");
+  t->map_kc = t->map_k; t->map_vc = t->map_vt;  // placeholders until a cache is supplied
+  if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return tfail(t, DC_ERR_CUDA, "cannot opt in to %d bytes of shared memory", kAttnSmem);
+  }
   cudaError_t e1 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_QKV>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kSmemBudget + 1024 - kStaticQkv);
@@ -229,7 +262,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   GemmParams p{};
   p.M = M; p.BN = BN; p.nq = nq; p.nkv = nkv; p.hd = hd;
   p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
-  p.q = t->q; p.k = t->k; p.v = t->v; p.act = t->act;
+  p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv; p.act = t->act;
   p.part = t->part; p.part_stride = t->part_stride;
 
   hook.begin(DC_STAGE_QKV, 1);
@@ -239,8 +272,26 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_ATTN, 1);
-  launch_attn_simt<__nv_bfloat16>(t->q, t->k, t->v, k_cache, v_cache, g.max_ctx, m, nq, nkv, hd,
-                                  t->o, t->s);
+  {
+    bool any_ctx = false;
+    for (int b = 0; b < m.batch; ++b) any_ctx |= m.ctx_len[b] > 0;
+    if (any_ctx && (t->kc_base != k_cache || t->vc_base != v_cache)) {
+      const uint64_t heads = (uint64_t)g.max_batch * nkv;
+      if (!(make_map_3d(&t->map_kc, k_cache, 128, heads * g.max_ctx, g.n_layers, 128) &&
+            make_map_3d(&t->map_vc, v_cache, g.max_ctx, heads * 128, g.n_layers, 128)))
+        return tfail(t, DC_ERR_CUDA, "cache tensor map encoding failed (caches must be 16-byte aligned)");
+      t->kc_base = k_cache; t->vc_base = v_cache;
+    }
+    AttnParams ap;
+    ap.m = m; ap.nq = nq; ap.nkv = nkv; ap.max_ctx = g.max_ctx; ap.layer = layer;
+    ap.scale_log2 = 1.4426950408889634f / sqrtf((float)hd);
+    ap.o = t->o; ap.status = t->status;
+    dim3 grid((m.R_cap + 127) / 128, nq, m.nv * m.batch);
+    k_attn_tc<<<grid, kAttnThreads, kAttnSmem, t->s>>>(t->map_q, t->map_k, t->map_vt, t->map_kc,
+                                                       t->map_vc, ap);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+  }
   hook.end();
 
   hook.begin(DC_STAGE_OPROJ, 1);

@@ -33,6 +33,7 @@ const char* tc_error(const TcState* t);
 // One transformer layer after the first RMSNorm: a = norm1(x) is given; on return the
 // attention and MLP residual updates are applied to x except for the split-K partial sums of
 // the last GEMM, which are handed back (part / nsplit / part_stride) for the next norm to fold.
+// k_cache / v_cache are the BASE pointers of the whole caches (all layers).
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,

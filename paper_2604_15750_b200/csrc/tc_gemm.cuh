@@ -34,7 +34,8 @@ struct GemmParams {
   int nq, nkv, hd;          // tiles [0,nq) are q heads, [nq,nq+nkv) k heads, rest v heads
   const float* cos_sin;     // RoPE table [(b, r)][hd]
   int rows_per_variant;     // batch * R_cap: the table is shared by the variants
-  __nv_bfloat16 *q, *k, *v; // outputs [M, nq*hd], [M, nkv*hd], [M, nkv*hd]
+  __nv_bfloat16 *q, *k, *v; // outputs q [M, nq*hd], k [M, nkv*hd], v TRANSPOSED [nkv*hd, ldv]
+  int ldv;                  // row pitch of the transposed v (elements, multiple of 8)
   // PARTIAL epilogue
   float* part;              // [nsplit][M_ld][N]
   size_t part_stride;       // elements between splits
@@ -193,12 +194,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         } else {  // GEMM_EPI_QKV
           const bool is_v = tile >= p.nq + p.nkv;
           if (is_v) {
-            __nv_bfloat16* dst = p.v + (size_t)((tile - p.nq - p.nkv) * p.hd + f);
-            const int ld = p.nkv * p.hd;
+            // V is stored transposed (keys contiguous): this thread's 32 columns are 32
+            // consecutive keys of feature row f
+            __nv_bfloat16* dst = p.v + (size_t)((tile - p.nq - p.nkv) * p.hd + f) * p.ldv + m_base + c0;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int m = m_base + c0 + j;
-              if (j < width && m < p.M) dst[(size_t)m * ld] = __float2bfloat16_rn(acc[j]);
+            for (int j = 0; j < 32; j += 8) {
+              if (j < width && m_base + c0 + j < p.M) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  __nv_bfloat162 pr = __floats2bfloat162_rn(acc[j + 2 * e], acc[j + 2 * e + 1]);
+                  w[e] = *reinterpret_cast<uint32_t*>(&pr);
+                }
+                *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
             }
           } else {
             // rotate-half RoPE: feature i < hd/2 pairs with i + hd/2, held by the warp two
