@@ -143,7 +143,8 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
   m->R_cap = round_up(maxR, 16);
   m->W_cap = round_up(maxW, 16);
   const int npos = batch * m->W_cap;
-  m->G = npos < 128 ? npos : 128;
+  const int gmax = 128 / m->nv;  // an LM-head group is [G curr rows ; G prev rows] <= 128 rows
+  m->G = npos < gmax ? npos : gmax;
   m->npos_pad = round_up(npos, m->G);
   return DC_OK;
 }
@@ -399,7 +400,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
   c->ws_lse = ws_alloc<float>(c, nw, &ok);
   if (c->use_tc) {
     int rc = tc_create(g, c->stream, c->M_max, c->Mlm_max, c->wq, c->wk, c->wv, c->wo, c->w_gate,
-                       c->w_up, c->w_down, c->lm_head, &c->tc);
+                       c->w_up, c->w_down, c->lm_head, (const __nv_bfloat16*)c->h, &c->tc);
     if (rc != DC_OK) {
       std::string why = c->tc ? tc_error(c->tc) : "tensor-core state allocation failed";
       dc_destroy(c);

@@ -10,6 +10,7 @@
 
 #include "tc_attn.cuh"
 #include "tc_gemm.cuh"
+#include "tc_lmhead.cuh"
 
 namespace dc {
 
@@ -90,6 +91,9 @@ struct TcState {
   int ldv = 0;  // row pitch of the transposed active V
   CUtensorMap map_q, map_k, map_vt, map_kc, map_vc;
   const void *kc_base = nullptr, *vc_base = nullptr;
+  CUtensorMap map_h, map_lm;
+  float* lm_part = nullptr;
+  int n_sm = 148, lm_stages = 6;
   std::string err;
   bool attrs_set = false;
 };
@@ -143,8 +147,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
               const std::vector<const void*>& wq, const std::vector<const void*>& wk,
               const std::vector<const void*>& wv, const std::vector<const void*>& wo,
               const std::vector<const void*>& w_gate, const std::vector<const void*>& w_up,
-              const std::vector<const void*>& w_down, const void* lm_head, TcState** out) {
-  (void)Mlm_max; (void)lm_head;
+              const std::vector<const void*>& w_down, const void* lm_head,
+              const __nv_bfloat16* h_buf, TcState** out) {
   TcState* t = new TcState();
   *out = t;
   t->g = g; t->s = s; t->M_max = M_max;
@@ -181,6 +185,26 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
         make_map_2d(&t->map_vt, t->v, hkv, t->ldv, 128)))
     return tfail(t, DC_ERR_CUDA, "attention tensor map encoding failed");
   t->map_kc = t->map_k; t->map_vc = t->map_vt;  // placeholders until a cache is supplied
+  {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&t->n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (t->n_sm < 1) t->n_sm = 148;
+    const size_t groups_max = ((size_t)g.max_batch * g.max_window + 63) / 64 + 1;
+    t->lm_part = talloc<float>(t, groups_max * t->n_sm * 128 * 8, &ok);
+    if (!ok) return tfail(t, DC_ERR_NOMEM, "LM-head workspace allocation failed");
+    if (!(make_map_2d(&t->map_h, h_buf, Mlm_max, d, 128) &&
+          make_map_2d(&t->map_lm, lm_head, g.vocab, d, 128)))
+      return tfail(t, DC_ERR_CUDA, "LM-head tensor map encoding failed");
+    const int lm_static = 2 * 64 * 33 * 4 + 512;
+    t->lm_stages = (kSmemBudget - lm_static) / kLmStageBytes;
+    if (t->lm_stages > 8) t->lm_stages = 8;
+    if (cudaFuncSetAttribute(k_lmhead_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             t->lm_stages * kLmStageBytes + 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return tfail(t, DC_ERR_CUDA, "cannot opt in to shared memory for the LM head");
+    }
+  }
   if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem) !=
       cudaSuccess) {
     cudaGetLastError();
@@ -321,10 +345,29 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   return DC_OK;
 }
 
-int tc_lmhead(TcState*, const SeqMeta&, const __nv_bfloat16*, int, int, int32_t*, float*, float*,
-              float*, float*, SignalOut) { return DC_ERR_UNSUPPORTED; }
+int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id, int forbid,
+              int32_t* ws_pred, float* ws_conf, float* ws_ent, float* ws_infl, float* ws_lse,
+              SignalOut out) {
+  (void)h;  // the tensor map was built over the scheduler's LM-head input buffer
+  const dc_config& g = t->g;
+  LmParams p;
+  p.m = m; p.V = g.vocab; p.K = g.d_model; p.mask_id = forbid ? mask_id : -1;
+  p.part = t->lm_part; p.status = t->status;
+  const int ntiles = (g.vocab + 127) / 128;
+  const int nctas = ntiles < t->n_sm ? ntiles : t->n_sm;
+  const int groups = m.npos_pad / m.G;
+  dim3 grid(nctas, groups);
+  k_lmhead_tc<<<grid, kLmThreads, t->lm_stages * kLmStageBytes + 1024, t->s>>>(t->map_h, t->map_lm,
+                                                                               p, t->lm_stages);
+  const int npos = m.batch * m.W_cap;
+  k_lm_combine<<<(npos + 3) / 4, 128, 0, t->s>>>(t->lm_part, nctas, m, ws_pred, ws_conf, ws_ent,
+                                                 ws_infl, ws_lse, out);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "LM-head launch failed: %s", cudaGetErrorString(e));
+  return DC_OK;
+}
 
-bool tc_has_lmhead(const dc_config&) { return false; }
+bool tc_has_lmhead(const dc_config& g) { return tc_supported(g); }
 
 __global__ void k_flush_status(int32_t* tc_status, int32_t* status, int batch) {
   if (*tc_status != 0) {

@@ -26,7 +26,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
               const std::vector<const void*>& wq, const std::vector<const void*>& wk,
               const std::vector<const void*>& wv, const std::vector<const void*>& wo,
               const std::vector<const void*>& w_gate, const std::vector<const void*>& w_up,
-              const std::vector<const void*>& w_down, const void* lm_head, TcState** out);
+              const std::vector<const void*>& w_down, const void* lm_head,
+              const __nv_bfloat16* h_buf, TcState** out);
 void tc_destroy(TcState* t);
 const char* tc_error(const TcState* t);
 

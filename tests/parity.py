@@ -100,13 +100,19 @@ class Case:
                                    else max(self.wl.last_len, 1), max_ctx=max_ctx)
         return eng
 
-    def device_inputs(self, eng):
+    def device_inputs(self, eng, poison=False):
         dev = eng.device
         B = self.wl.batch
         kc = vc = None
         if self.k_log is not None:
             kc, vc = pack_kv_cache(self.k_log.to(dev), self.v_log.to(dev), eng.max_batch,
                                    eng.max_ctx)
+            if poison:      # the cache beyond ctx_len may hold anything, NaN included
+                for b in range(B):
+                    P = self.len["ctx_len"][b]
+                    kc[:, b, :, P:, :] = float("nan")
+                    vc[:, b, :, :, P:] = float("nan")
+                kc[:, B:] = float("nan"); vc[:, B:] = float("nan")
         last = torch.zeros((B, eng.max_last), dtype=torch.int32)
         last[:, :self.last_ids.shape[1]] = self.last_ids
         win = torch.full((B, eng.max_window), self.wl.mask_id, dtype=torch.int32)
@@ -120,8 +126,8 @@ class Case:
                     last_len=self.len["last_len"], win_ids=win.to(dev),
                     win_len=self.len["win_len"], remain_len=self.len["remain_len"], h_final=hf)
 
-    def run_gpu(self, eng, influence=True, boundary=True):
-        di = self.device_inputs(eng)
+    def run_gpu(self, eng, influence=True, boundary=True, poison=False):
+        di = self.device_inputs(eng, poison)
         out = eng.step(influence=influence, boundary=boundary, **di)
         sel = eng.select(di["win_ids"], di["win_len"])
         eng.synchronize()

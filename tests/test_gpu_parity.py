@@ -51,7 +51,7 @@ def test_small_bf16_ragged_batch_grouped_heads_mid_block():
                    remain_len=[64, 17, 30])
     case = Case(SMALL_BF16, lengths=lengths, n_decoded=4)
     eng = case.make_engine()
-    gpu, ora = case.run_gpu(eng), case.run_oracle()
+    gpu, ora = case.run_gpu(eng, poison=True), case.run_oracle()
     near, worst = compare(case, gpu, ora)
     assert int(gpu["block_len"][2]) == min(8, 9)          # sequence 2 has no last block
     assert np.all(gpu["influence"][2, :9] == 0)

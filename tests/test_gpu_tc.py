@@ -55,3 +55,24 @@ def test_tc_and_cuda_core_paths_agree():
     assert np.abs(a["lse"][:2, :W] - b["lse"][:2, :W]).max() < 2e-2
     assert np.array_equal(a["pred_id"][:2, :W], b["pred_id"][:2, :W])
     e1.close(); e2.close()
+
+
+def test_tc_cache_beyond_ctx_len_may_hold_nan():
+    wl = _wl(3)
+    lengths = dict(ctx_len=[128, 41, 7], last_len=[16, 16, 3], win_len=[32, 30, 32],
+                   remain_len=[64, 64, 64])
+    case = Case(wl, lengths=lengths)
+    eng = case.make_engine(max_batch=4, max_ctx=192)
+    gpu, ora = case.run_gpu(eng, poison=True), case.run_oracle()
+    compare(case, gpu, ora)
+    eng.close()
+
+
+def test_tc_more_than_128_active_rows_and_long_context():
+    """R = 32 + 128 = 160 active rows: two query tiles and two active key tiles; 5 context tiles."""
+    wl = _wl(2, ctx=(513, 600), last=32, win=128)
+    case = Case(wl)
+    eng = case.make_engine()
+    gpu, ora = case.run_gpu(eng, poison=True), case.run_oracle()
+    compare(case, gpu, ora)
+    eng.close()
