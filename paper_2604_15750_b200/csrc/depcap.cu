@@ -330,6 +330,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
       g.d_ff < 1 || g.vocab < 2)
     return fail(nullptr, DC_ERR_INVALID_ARG, "non-positive model dimension");
   if (g.head_dim % 2) return fail(nullptr, DC_ERR_INVALID_ARG, "head_dim must be even");
+  if (g.d_model % 4) return fail(nullptr, DC_ERR_UNSUPPORTED, "d_model must be a multiple of 4");
   if (g.n_q_heads % g.n_kv_heads)
     return fail(nullptr, DC_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
   if (g.mask_id < 0 || g.mask_id >= g.vocab)

@@ -76,25 +76,67 @@ void launch_embed(const T* embed, const int32_t* last_ids, const int32_t* win_id
 }
 
 // ---- RMSNorm (with the split-K partial sums of the preceding GEMM folded into x) --------------
+template <typename T> __device__ __forceinline__ void store4(T* dst, const float (&v)[4]);
+template <> __device__ __forceinline__ void store4<float>(float* dst, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* dst,
+                                                                   const float (&v)[4]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(dst) =
+      make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+template <typename T> __device__ __forceinline__ void load4(const T* src, float (&v)[4]);
+template <> __device__ __forceinline__ void load4<float>(const float* src, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(src);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* src,
+                                                                  float (&v)[4]) {
+  const uint2 t = *reinterpret_cast<const uint2*>(src);
+  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+  v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
+}
+
+// One row per block; d is a multiple of 4.  The row (with the partial sums folded in, in split
+// order, so the result does not depend on the launch shape) is written back to x and normed.
 template <typename T>
-__global__ void k_rmsnorm(float* __restrict__ x, const float* __restrict__ part, int nsplit,
-                          size_t part_stride, const T* __restrict__ g, float eps, int d,
-                          T* __restrict__ out) {
-  __shared__ float red[32];
-  const size_t off = (size_t)blockIdx.x * d;
+__device__ __forceinline__ void rmsnorm_row(float* __restrict__ xr, const float* __restrict__ part,
+                                            int nsplit, size_t part_stride, const T* __restrict__ g,
+                                            float eps, int d, T* __restrict__ outr, float* red) {
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = x[off + i];
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(xr + i);
     if (part) {
-      for (int sidx = 0; sidx < nsplit; ++sidx) v += part[sidx * part_stride + off + i];
-      x[off + i] = v;
+      for (int sidx = 0; sidx < nsplit; ++sidx) {
+        const float4 pv = *reinterpret_cast<const float4*>(part + sidx * part_stride + i);
+        v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
+      }
+      *reinterpret_cast<float4*>(xr + i) = v;
     }
-    ss += v * v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, red);
   const float inv = rsqrtf(ss / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    out[off + i] = from_f<T>(x[off + i] * inv * to_f<T>(g[i]));
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(xr + i);
+    float gv[4];
+    load4<T>(g + i, gv);
+    const float o[4] = {v.x * inv * gv[0], v.y * inv * gv[1], v.z * inv * gv[2], v.w * inv * gv[3]};
+    store4<T>(outr + i, o);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ x,
+                                                 const float* __restrict__ part, int nsplit,
+                                                 size_t part_stride, const T* __restrict__ g,
+                                                 float eps, int d, T* __restrict__ out) {
+  __shared__ float red[32];
+  const size_t off = (size_t)blockIdx.x * d;
+  rmsnorm_row<T>(x + off, part ? part + off : nullptr, nsplit, part_stride, g, eps, d, out + off,
+                 red);
 }
 
 template <typename T>
@@ -119,19 +161,7 @@ __global__ void k_final_norm(float* __restrict__ x, const float* __restrict__ pa
     return;
   }
   const size_t off = (size_t)act_row(m, v, b, m.last_len[b] + k) * d;
-  float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float val = x[off + i];
-    if (part) {
-      for (int sidx = 0; sidx < nsplit; ++sidx) val += part[sidx * part_stride + off + i];
-      x[off + i] = val;
-    }
-    ss += val * val;
-  }
-  ss = block_sum(ss, red);
-  const float inv = rsqrtf(ss / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    hr[i] = from_f<T>(x[off + i] * inv * to_f<T>(g[i]));
+  rmsnorm_row<T>(x + off, part ? part + off : nullptr, nsplit, part_stride, g, eps, d, hr, red);
 }
 
 template <typename T>

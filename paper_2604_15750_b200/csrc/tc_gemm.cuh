@@ -222,14 +222,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
             __nv_bfloat16* dst = is_k ? p.k + (size_t)((tile - p.nq) * p.hd + f)
                                       : p.q + (size_t)(tile * p.hd + f);
             const int ld = is_k ? p.nkv * p.hd : p.nq * p.hd;
+            // all table reads of the chunk first (independent loads), then the rotation
+            float cv[32], sv[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              int m = m_base + c0 + j;
+              if (m >= p.rows_per_variant) m -= p.rows_per_variant;  // prev variant: same table
+              const bool in = j < width && m_base + c0 + j < p.M;
+              const float* cs = p.cos_sin + (size_t)(in ? m : 0) * p.hd;
+              cv[j] = __ldg(cs + i);
+              sv[j] = __ldg(cs + half + i);
+            }
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int m = m_base + c0 + j;
               if (j < width && m < p.M) {
                 const float other = xch[(f ^ half) * 33 + j];
-                const float* cs = p.cos_sin + (size_t)(m % p.rows_per_variant) * p.hd;
-                const float c = cs[i], sn = cs[half + i];
-                const float y = lo ? (acc[j] * c - other * sn) : (acc[j] * c + other * sn);
+                const float y = lo ? (acc[j] * cv[j] - other * sv[j]) : (acc[j] * cv[j] + other * sv[j]);
                 dst[(size_t)m * ld] = __float2bfloat16_rn(y);
               }
             }

@@ -176,17 +176,28 @@ def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
             worst["xlogp"] = max(worst["xlogp"], float(e))
             assert e <= rtol, ("xlogp", b, e)
         # ---- block length
-        if check_boundary:
+        if check_boundary and len(o["score"]):
+            # The score divides I and H by their window maxima, so an input error dI becomes
+            # dI / max(I) in the score (random-init weights give I ~ 1e-5, where fp32 rounding of
+            # the KL sum is already visible).  Bound the score error by the observed input errors.
+            n = len(o["score"])
+            dI = np.abs(gpu["influence"][b, :n] - o["influence"][:n]).max()
+            dH = np.abs(gpu["entropy"][b, :n] - o["entropy"][:n]).max()
+            Imax = max(float(np.max(o["influence"][:n])), 1e-8)
+            Hmax = max(float(np.max(o["entropy"][:n])), 1e-8)
+            if hp.norm_mode == 2:
+                Imax = Hmax = 1.0
+            sbound = 4.0 * (dI / Imax + hp.lam * dH / Hmax) + 1e-5
             Lg, Lo = int(gpu["block_len"][b]), int(o["block_len"])
             if Lg != Lo:
                 lo, hi = min(Lg, Lo), max(Lg, Lo)
-                s = o["score"][:hi + 1]
-                assert np.abs(s[lo:]).min() <= rtol or \
-                    np.abs(o["cum_score"][lo:hi + 1]).min() <= rtol * max(1, hi), (b, Lg, Lo)
+                s_ = o["score"][:hi + 1]
+                assert np.abs(s_[lo:]).min() <= sbound or \
+                    np.abs(o["cum_score"][lo:hi + 1]).min() <= sbound * max(1, hi), (b, Lg, Lo)
                 near["block_len"] += 1
-            else:
-                n = len(o["score"])
-                assert np.allclose(gpu["score"][b, :n], o["score"], atol=2 * rtol, rtol=rtol)
+            elif o["influence"][:n].max() > 0:
+                assert np.abs(gpu["score"][b, :n] - o["score"]).max() <= sbound, \
+                    (b, np.abs(gpu["score"][b, :n] - o["score"]).max(), sbound)
         # ---- selected subset
         cnt = int(gpu["sel_count"][b])
         sel_g = sorted(int(i) for i in gpu["sel_idx"][b, :cnt])
