@@ -326,7 +326,7 @@ def main():
         return
 
     peaks = _peaks()
-    gemm_ms = sum(stage_ms[n] for n in ("qkv", "oproj", "gateup", "down"))
+    gemm_ms = sum(stage_ms[n] for n in ("qkv", "oproj", "gateup", "down", "dense"))
     M = 2 * wl.batch * ((wl.last_len + wl.win_len + 15) // 16 * 16)
     w_bytes = 2.0 * _layer_param_count(wl) * n_layers
     flops = 2.0 * _layer_param_count(wl) * n_layers * M

@@ -232,6 +232,7 @@ DC_API int dc_debug_logits(dc_ctx* ctx, int32_t variant, float* out);
 /* Per-stage device time of the last dc_step_profiled call, in milliseconds. */
 enum { DC_STAGE_EMBED = 0, DC_STAGE_NORM, DC_STAGE_QKV, DC_STAGE_ATTN, DC_STAGE_OPROJ,
        DC_STAGE_GATEUP, DC_STAGE_DOWN, DC_STAGE_LMHEAD, DC_STAGE_XLOGP, DC_STAGE_BOUNDARY,
+       DC_STAGE_DENSE, /* fused launch: O projection, norms, gate/up, down, QKV of the next layer */
        DC_STAGE_COUNT };
 
 /* dc_step with CUDA events around every stage; synchronises the stream before returning and

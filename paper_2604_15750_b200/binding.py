@@ -16,7 +16,7 @@ DC_F32, DC_BF16 = 0, 1
 DC_STEP_INFLUENCE, DC_STEP_BOUNDARY = 1, 2
 DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
-               "boundary"]
+               "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
            "dc_debug_logits", "dc_step_profiled"]
 

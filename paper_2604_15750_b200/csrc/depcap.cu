@@ -183,7 +183,36 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
   int nsplit = 0;
   size_t part_stride = 0;
 
-  for (int l = 0; l < g.n_layers; ++l) {
+  const bool chain = c->use_tc && tc_chain_ok(c->tc, m);
+  if (c->use_tc) tc_step_begin(c->tc);
+  if (chain) {
+    // persistent dense chain: norm1 + QKV of layer 0, then per layer attention and one launch
+    // that runs O projection .. QKV of the next layer
+    const int L = g.n_layers;
+    pf.begin(DC_STAGE_DENSE, 1);
+    int rc = tc_chain(c->tc, 0, 0, CH_NORM1, CH_END, m, c->x, (const __nv_bfloat16*)a, c->cos_sin,
+                      nullptr, (const __nv_bfloat16*)c->norm1[0], 0, &part, &nsplit, &part_stride);
+    pf.end();
+    if (rc != DC_OK) return fail(c, rc, "dense chain failed: %s", tc_error(c->tc));
+    for (int l = 0; l < L; ++l) {
+      pf.begin(DC_STAGE_ATTN, 1);
+      rc = tc_attention(c->tc, l, m, (const __nv_bfloat16*)in->k_cache,
+                        (const __nv_bfloat16*)in->v_cache);
+      pf.end();
+      if (rc != DC_OK) return fail(c, rc, "attention failed: %s", tc_error(c->tc));
+      const bool last = l + 1 == L;
+      pf.begin(DC_STAGE_DENSE, 1);
+      rc = tc_chain(c->tc, l, l + 1, CH_OPROJ, last ? CH_NORM1 : CH_END, m, c->x,
+                    (const __nv_bfloat16*)a, c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
+                    last ? nullptr : (const __nv_bfloat16*)c->norm1[l + 1], nsplit, &part, &nsplit,
+                    &part_stride);
+      pf.end();
+      if (rc != DC_OK) return fail(c, rc, "dense chain failed: %s", tc_error(c->tc));
+    }
+    DC_CHECK_LAUNCH(c);
+  }
+
+  for (int l = 0; l < g.n_layers && !chain; ++l) {
     pf.begin(DC_STAGE_NORM, 1);
     launch_rmsnorm<T>(c->x, part, nsplit, part_stride, (const T*)c->norm1[l], g.rms_eps, M, d, a, s);
     pf.end();

@@ -4,11 +4,14 @@
 #include <cuda.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include <map>
 #include <string>
 
 #include "tc_attn.cuh"
+#include "tc_chain.cuh"
 #include "tc_gemm.cuh"
 #include "tc_lmhead.cuh"
 
@@ -94,6 +97,8 @@ struct TcState {
   CUtensorMap map_h, map_lm;
   float* lm_part = nullptr;
   int n_sm = 148, lm_stages = 6;
+  unsigned int* grid_bar = nullptr;  // {count, generation} of the dense chain's grid barrier
+  int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
   std::string err;
   bool attrs_set = false;
 };
@@ -223,6 +228,23 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
     cudaGetLastError();
     return tfail(t, DC_ERR_CUDA, "cannot opt in to %d bytes of shared memory", kSmemBudget);
   }
+  // the persistent dense chain needs every CTA resident at once (cooperative launch)
+  {
+    t->grid_bar = talloc<unsigned int>(t, 2, &ok);
+    if (!ok) return tfail(t, DC_ERR_NOMEM, "dense-chain workspace allocation failed");
+    cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), s);
+    int dev = 0, coop = 0, per_sm = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (coop &&
+        cudaFuncSetAttribute(k_dense_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem) ==
+            cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_dense_chain, kChainThreads, kChainSmem) ==
+            cudaSuccess &&
+        per_sm >= 1)
+      t->chain_grid = t->n_sm;
+    cudaGetLastError();
+  }
   return DC_OK;
 }
 
@@ -271,6 +293,112 @@ static int pick_split(int tiles, int KB, int max_split) {
   return s;
 }
 
+int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,
+                 const __nv_bfloat16* v_cache) {
+  const dc_config& g = t->g;
+  const int nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim;
+  bool any_ctx = false;
+  for (int b = 0; b < m.batch; ++b) any_ctx |= m.ctx_len[b] > 0;
+  if (any_ctx && (t->kc_base != k_cache || t->vc_base != v_cache)) {
+    const uint64_t heads = (uint64_t)g.max_batch * nkv;
+    if (!(make_map_3d(&t->map_kc, k_cache, 128, heads * g.max_ctx, g.n_layers, 128) &&
+          make_map_3d(&t->map_vc, v_cache, g.max_ctx, heads * 128, g.n_layers, 128)))
+      return tfail(t, DC_ERR_CUDA, "cache tensor map encoding failed (caches must be 16-byte aligned)");
+    t->kc_base = k_cache; t->vc_base = v_cache;
+  }
+  AttnParams ap;
+  ap.m = m; ap.nq = nq; ap.nkv = nkv; ap.max_ctx = g.max_ctx; ap.layer = layer;
+  ap.scale_log2 = 1.4426950408889634f / sqrtf((float)hd);
+  ap.o = t->o; ap.status = t->status;
+  dim3 grid((m.R_cap + 127) / 128, nq, m.nv * m.batch);
+  k_attn_tc<<<grid, kAttnThreads, kAttnSmem, t->s>>>(t->map_q, t->map_k, t->map_vt, t->map_kc,
+                                                     t->map_vc, ap);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+  return DC_OK;
+}
+
+bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
+  const int M = m.nv * m.batch * m.R_cap;
+  // one column block of at most 256 activation rows; the ring must hold two gate/up stages
+  return t->chain_grid > 0 && M <= 256;
+}
+
+void tc_step_begin(TcState* t) {
+  // a step that gave up inside a grid barrier leaves the arrival count behind
+  cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), t->s);
+}
+
+int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_end, const SeqMeta& m,
+             float* x, const __nv_bfloat16* a, const float* cos_sin, const __nv_bfloat16* g2,
+             const __nv_bfloat16* g1, int fold_norm1, const float** part, int* nsplit,
+             size_t* part_stride) {
+  const dc_config& g = t->g;
+  const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, F = g.d_ff;
+  const int M = m.nv * m.batch * m.R_cap;
+  const int BN = (M + 15) / 16 * 16;
+  ActMaps* am = nullptr;
+  int rc = get_act_maps(t, a, BN, &am);
+  if (rc != DC_OK) return rc;
+  ChainMaps maps;
+  const LayerMaps& L = t->layers[layer];
+  const LayerMaps& Lq = t->layers[qkv_layer < g.n_layers ? qkv_layer : layer];
+  maps.wo = L.wo; maps.wg = L.w_gate; maps.wu = L.w_up; maps.wd = L.w_down;
+  maps.wq = Lq.wq; maps.wk = Lq.wk; maps.wv = Lq.wv;
+  maps.a = am->a; maps.o = am->o; maps.act = am->act;
+  ChainParams p{};
+  p.M = M; p.BN = BN; p.d = d; p.F = F; p.nq = nq; p.nkv = nkv;
+  p.phase_begin = phase_begin; p.phase_end = phase_end;
+  p.split_o = pick_split(d / kChainTile, nq * g.head_dim / kChainTileK, t->max_split);
+  p.split_down = pick_split(d / kChainTile, F / kChainTileK, t->max_split);
+  p.fold_norm1 = fold_norm1;
+  p.x = x; p.a = const_cast<__nv_bfloat16*>(a); p.act = t->act;
+  p.part = t->part; p.part_stride = t->part_stride;
+  p.g2 = g2; p.g1 = g1; p.eps = g.rms_eps;
+  p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
+  p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv;
+  p.bar = t->grid_bar; p.status = t->status;
+#ifdef DC_CHAIN_TRACE
+  static unsigned long long* trace_buf = nullptr;
+  static unsigned long long* trace_dev = nullptr;
+  if (!trace_buf) {
+    trace_buf = (unsigned long long*)malloc(256 * 64 * sizeof(unsigned long long));
+    cudaMalloc(&trace_dev, 256 * 64 * sizeof(unsigned long long));
+  }
+  cudaMemsetAsync(trace_dev, 0, 256 * 64 * sizeof(unsigned long long), t->s);
+  p.trace = trace_dev;
+#endif
+  void* args[] = {&maps, &p};
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)k_dense_chain, dim3(t->chain_grid),
+                                              dim3(kChainThreads), args, kChainSmem, t->s);
+#ifdef DC_CHAIN_TRACE
+  {
+    static int n_print = 0;
+    if (layer == 5 && n_print < 3) {
+      cudaStreamSynchronize(t->s);
+      cudaMemcpy(trace_buf, trace_dev, 256 * 64 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+      ++n_print;
+      char fn[64];
+      snprintf(fn, sizeof(fn), "gpurun_out/chain_trace_dbg0_%d.txt", n_print);
+      FILE* f = fopen(fn, "w");
+      if (f) {
+        for (int c = 0; c < t->chain_grid; ++c) {
+          for (int i = 0; i < 64; ++i) fprintf(f, "%llu ", trace_buf[c * 64 + i]);
+          fprintf(f, "\n");
+        }
+        fclose(f);
+      }
+    }
+  }
+#endif
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return tfail(t, DC_ERR_CUDA, "dense chain launch failed: %s", cudaGetErrorString(e));
+  }
+  *part = t->part; *nsplit = p.split_down; *part_stride = t->part_stride;
+  return DC_OK;
+}
+
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
@@ -296,27 +424,9 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_ATTN, 1);
-  {
-    bool any_ctx = false;
-    for (int b = 0; b < m.batch; ++b) any_ctx |= m.ctx_len[b] > 0;
-    if (any_ctx && (t->kc_base != k_cache || t->vc_base != v_cache)) {
-      const uint64_t heads = (uint64_t)g.max_batch * nkv;
-      if (!(make_map_3d(&t->map_kc, k_cache, 128, heads * g.max_ctx, g.n_layers, 128) &&
-            make_map_3d(&t->map_vc, v_cache, g.max_ctx, heads * 128, g.n_layers, 128)))
-        return tfail(t, DC_ERR_CUDA, "cache tensor map encoding failed (caches must be 16-byte aligned)");
-      t->kc_base = k_cache; t->vc_base = v_cache;
-    }
-    AttnParams ap;
-    ap.m = m; ap.nq = nq; ap.nkv = nkv; ap.max_ctx = g.max_ctx; ap.layer = layer;
-    ap.scale_log2 = 1.4426950408889634f / sqrtf((float)hd);
-    ap.o = t->o; ap.status = t->status;
-    dim3 grid((m.R_cap + 127) / 128, nq, m.nv * m.batch);
-    k_attn_tc<<<grid, kAttnThreads, kAttnSmem, t->s>>>(t->map_q, t->map_k, t->map_vt, t->map_kc,
-                                                       t->map_vc, ap);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
-  }
+  rc = tc_attention(t, layer, m, k_cache, v_cache);
   hook.end();
+  if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_OPROJ, 1);
   p.N = d; p.K = nq * hd; p.nsplit = pick_split(d / kTileN, p.K / kTileK, t->max_split);

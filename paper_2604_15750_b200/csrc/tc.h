@@ -15,6 +15,9 @@ struct StageHook {
 
 struct TcState;
 
+// phases of the persistent dense chain, in execution order
+enum { CH_OPROJ = 0, CH_NORM2 = 1, CH_GATEUP = 2, CH_DOWN = 3, CH_NORM1 = 4, CH_QKV = 5, CH_END = 6 };
+
 // true if the tensor-core kernels take this model shape
 bool tc_supported(const dc_config& g);
 // true if the fused tensor-core LM head takes this model shape
@@ -39,6 +42,23 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
              StageHook& hook);
+
+// Attention of one layer alone (reads the rotated q / k / transposed v the QKV epilogue wrote).
+int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,
+                 const __nv_bfloat16* v_cache);
+
+// true if the persistent dense chain takes this step (all activation rows in one column block)
+bool tc_chain_ok(const TcState* t, const SeqMeta& m);
+// resets the chain's grid barrier; call once at the start of a step
+void tc_step_begin(TcState* t);
+// Phases [phase_begin, phase_end) of the dense chain (CH_* in tc_chain.cuh): O projection,
+// residual + norm2 (gain g2), gate/up, down projection of `layer`; residual + norm1 (gain g1,
+// folding fold_norm1 partial sums) and the rotated QKV of `qkv_layer`.  The partial sums of the
+// last GEMM that ran are handed back like tc_layer does.
+int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_end, const SeqMeta& m,
+             float* x, const __nv_bfloat16* a, const float* cos_sin, const __nv_bfloat16* g2,
+             const __nv_bfloat16* g1, int fold_norm1, const float** part, int* nsplit,
+             size_t* part_stride);
 
 // LM head fused with the streaming softmax statistics; fills the workspace signal arrays and
 // the caller's outputs.  Never writes logits.

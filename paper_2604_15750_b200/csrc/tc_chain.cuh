@@ -1,0 +1,494 @@
+// Persistent dense chain: everything of a transformer layer between two attention calls, in one
+// cooperative launch with one CTA per SM.
+//
+//   phase 0  O projection        split-K partial sums of  o . Wo^T                (tcgen05)
+//   phase 1  residual + norm2    x += sum of partials;  a = bf16(rmsnorm(x) * g2)
+//   phase 2  gate / up           act = bf16(silu(a . Wg^T) * (a . Wu^T))          (tcgen05)
+//   phase 3  down projection     split-K partial sums of  act . Wd^T              (tcgen05)
+//   phase 4  residual + norm1    x += sum of partials;  a = bf16(rmsnorm(x) * g1') (next layer)
+//   phase 5  QKV of the next layer, rotated (RoPE), q / k row-major, v transposed  (tcgen05)
+//
+// A launch runs the phases [phase_begin, phase_end); CTAs meet at a grid-wide barrier between
+// phases.  The first layer starts with a launch of phases 4..5, the last layer ends after phase 3
+// (the final norm folds its partial sums).
+//
+// Why one kernel: at 192 activation rows a layer is 436 MB of weights (67 us of HBM time) cut
+// into four GEMMs of 5..30 us each; as separate launches every one of them pays its own launch,
+// pipeline ramp, and an epilogue that nothing overlaps.  Here the weight stream of the next phase
+// is already on its way into L2 (cp.async.bulk.prefetch) while the current phase drains, and the
+// only cost between phases is the barrier.
+//
+// GEMM orientation (as in tc_gemm.cuh): a CTA owns 128 weight rows (MMA M, one TMEM lane per
+// output feature) and all activation rows (MMA N <= 256, one TMEM column per row).  Every unit
+// keeps TWO accumulators in flight, because a chain of tcgen05.mma into one accumulator issues
+// at 151 clk per MMA while two alternating accumulators reach max(86, N/2 + 21) clk: gate / up
+// use one accumulator each, the other GEMMs send even k-steps to the first and odd k-steps to the
+// second and add them in the epilogue.
+//
+// Warp roles (192 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
+// owns the TMEM allocation), warps 2..5 = epilogue.  All six warps run the norm phases.
+#pragma once
+#include "kernels.h"
+#include "tc.h"
+#include "tc_ptx.cuh"
+
+namespace dc {
+
+struct ChainMaps {
+  CUtensorMap wo, wg, wu, wd;   // this layer: [d, hq], [F, d], [F, d], [d, F]
+  CUtensorMap wq, wk, wv;       // the layer whose QKV phase 5 computes
+  CUtensorMap a, o, act;        // activation operands, box = BN rows x 64 columns
+};
+
+struct ChainParams {
+  int M, BN;                    // valid activation rows; rows per MMA (multiple of 16, <= 256)
+  int d, F, nq, nkv;            // model width, MLP width, query / kv heads (head_dim 128)
+  int phase_begin, phase_end;
+  int split_o, split_down;      // split-K factors of the two projections back to d
+  int fold_norm1;               // partial sums phase 4 folds (0 when the launch starts there)
+  float* x;                     // residual stream [M, d] fp32
+  __nv_bfloat16* a;             // normed activations [M, d]
+  __nv_bfloat16* act;           // SwiGLU output [M, F]
+  float* part;                  // split-K partial sums [split][M][d]
+  size_t part_stride;
+  const __nv_bfloat16* g2;      // norm2 gain of this layer
+  const __nv_bfloat16* g1;      // norm1 gain of the layer phase 5 belongs to
+  float eps;
+  const float* cos_sin;         // RoPE table [(b, r)][128]
+  int rows_per_variant;
+  __nv_bfloat16 *q, *k, *v;     // q [M, nq*128], k [M, nkv*128], v transposed [nkv*128, ldv]
+  int ldv;
+  unsigned int* bar;            // grid barrier words {count, generation}
+  int32_t* status;              // DC_ERR_TIMEOUT lands here; non-zero on entry = do nothing
+#ifdef DC_CHAIN_TRACE
+  unsigned long long* trace;    // [cta][16] globaltimer at phase boundaries (tracing build only)
+#endif
+};
+
+constexpr int kChainThreads = 192;
+constexpr int kChainRing = 208 * 1024;          // TMA ring
+constexpr int kChainXch = 128 * 17 * 4;         // RoPE exchange buffer of the QKV epilogue
+constexpr int kChainSmem = kChainRing + kChainXch + 1024;
+constexpr int kChainTile = 128;                 // weight rows per unit
+constexpr int kChainTileK = 64;
+constexpr int kPrefetchAhead = 8;              // k-blocks the L2 prefetch runs ahead of the TMA loads
+
+struct ChainCtx {
+  uint8_t* ring;
+  float* xch;
+  uint64_t *full, *empty, *acc_full, *acc_empty;
+  volatile int* abort_flag;
+  uint32_t tmem_base;
+  uint32_t fill_bits;   // producer: parity of the next fill of each slot
+  uint32_t use_bits;    // MMA issuer: parity of the next use of each slot
+  uint32_t units_done;  // accumulator hand-overs so far (MMA issuer and epilogue count alike)
+  int warp, lane;
+};
+
+struct GemmPhase {
+  const CUtensorMap *w0, *w1, *w2;  // weight maps (QKV: q, k, v;  gate/up: gate, up)
+  const CUtensorMap* amap;          // activation operand
+  int tiles;                        // 128-row weight tiles (over all matrices of the phase)
+  int nsplit;                       // K splits
+  int KB;                           // k-blocks of 64
+  int N;                            // output features (row pitch of the output)
+  // what the producer prefetches into L2 once its own loads are issued: the first pf_kb
+  // k-blocks of its unit in the phase named here (tiles == 0: nothing)
+  const CUtensorMap *pf_w0, *pf_w1, *pf_w2;
+  int pf_tiles, pf_nsplit, pf_KB, pf_kb, pf_t1, pf_t2;  // pf_t1 / pf_t2: first tile of w1 / w2
+};
+
+// Loads, MMAs and epilogue of one GEMM phase.  Every thread of the CTA calls it.
+enum { CEPI_PARTIAL = 0, CEPI_SWIGLU = 1, CEPI_QKV = 2 };
+
+// Epilogue of 16 accumulator columns (activation rows c0 .. c0+15) of feature f of a tile.
+template <int EPI>
+__device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, const int N,
+                                           const int tile, const int split, const int f,
+                                           const int c0, float (&v0)[16], float (&v1)[16]) {
+  if (EPI == CEPI_PARTIAL) {
+    float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kChainTile + f) +
+                 (size_t)c0 * N;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) dst[(size_t)j * N] = v0[j] + v1[j];
+  } else if (EPI == CEPI_SWIGLU) {
+    __nv_bfloat16* dst = p.act + (size_t)(tile * kChainTile + f) + (size_t)c0 * N;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float gt = v0[j];
+      dst[(size_t)j * N] = __float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * v1[j]);
+    }
+  } else {  // CEPI_QKV
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v0[j] += v1[j];
+    const bool is_v = tile >= p.nq + p.nkv;
+    if (is_v) {
+      // V is stored transposed (keys contiguous): 16 consecutive keys of feature row f
+      __nv_bfloat16* dst = p.v + (size_t)((tile - p.nq - p.nkv) * 128 + f) * p.ldv + c0;
+#pragma unroll
+      for (int j = 0; j < 16; j += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 pr = __floats2bfloat162_rn(v0[j + 2 * e], v0[j + 2 * e + 1]);
+          w[e] = *reinterpret_cast<uint32_t*>(&pr);
+        }
+        *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    } else {
+      // rotate-half RoPE: feature i < 64 pairs with i + 64, held by the warp two quarters
+      // away; the chunk is exchanged through shared memory
+#pragma unroll
+      for (int j = 0; j < 16; ++j) c.xch[f * 17 + j] = v0[j];
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int i = f & 63;
+      const bool lo = f < 64;
+      const bool is_k = tile >= p.nq;
+      const int ld = is_k ? p.nkv * 128 : p.nq * 128;
+      __nv_bfloat16* dst = (is_k ? p.k + (size_t)((tile - p.nq) * 128 + f)
+                                 : p.q + (size_t)(tile * 128 + f)) + (size_t)c0 * ld;
+      int m0 = c0;  // a chunk of 16 rows never straddles the variants (rows_per_variant % 16 == 0)
+      if (m0 >= p.rows_per_variant) m0 -= p.rows_per_variant;  // prev variant: same table
+      const float* cs = p.cos_sin + (size_t)m0 * 128 + i;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float cv = __ldg(cs + j * 128), sv = __ldg(cs + j * 128 + 64);
+        const float other = c.xch[(f ^ 64) * 17 + j];
+        const float y = lo ? (v0[j] * cv - other * sv) : (v0[j] * cv + other * sv);
+        dst[(size_t)j * ld] = __float2bfloat16_rn(y);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+  }
+}
+
+#ifdef DC_CHAIN_TRACE
+#define DC_TRACE(slot) p.trace[blockIdx.x * 64 + 16 + (ph) * 4 + (slot)] = ptx::globaltimer()
+#else
+#define DC_TRACE(slot)
+#endif
+
+template <int EPI>
+__device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, const GemmPhase& g,
+                                           const int ph) {
+  constexpr int NW = (EPI == CEPI_SWIGLU) ? 2 : 1;
+  const int BN = p.BN;
+  const int slot_bytes = NW * kChainTile * kChainTileK * 2 + BN * kChainTileK * 2;
+  int stages = kChainRing / slot_bytes;
+  if (stages > 8) stages = 8;
+  const int n_units = g.tiles * g.nsplit;
+
+  if (c.warp == 0) {
+    if (c.lane == 0) {
+      // ---------------- TMA producer ----------------
+      bool ok = true;
+      int it = 0;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int tile = u / g.nsplit, split = u % g.nsplit;
+        const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
+        const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
+        const CUtensorMap* mw = g.w0;
+        int wrow = tile * kChainTile;
+        if (EPI == CEPI_QKV) {
+          if (tile >= p.nq + p.nkv) { mw = g.w2; wrow = (tile - p.nq - p.nkv) * kChainTile; }
+          else if (tile >= p.nq) { mw = g.w1; wrow = (tile - p.nq) * kChainTile; }
+        }
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % stages;
+          const uint32_t par = (c.fill_bits >> s) & 1u;
+          c.fill_bits ^= 1u << s;
+          ok = ptx::mbar_wait(&c.empty[s], par ^ 1u, c.abort_flag);
+          if (!ok) break;
+          uint8_t* slot = c.ring + (size_t)s * slot_bytes;
+          ptx::mbar_expect_tx(&c.full[s], (uint32_t)slot_bytes);
+          const int kc = kb * kChainTileK;
+          // keep the HBM -> L2 stream kPrefetchAhead k-blocks ahead of the shared-memory ring:
+          // the ring alone (3..5 slots) cannot cover the HBM latency at full bandwidth
+          if (kb + kPrefetchAhead < kb1) {
+            ptx::tma_prefetch_l2_2d(mw, kc + kPrefetchAhead * kChainTileK, wrow);
+            if (NW == 2) ptx::tma_prefetch_l2_2d(g.w1, kc + kPrefetchAhead * kChainTileK, wrow);
+          }
+          ptx::tma_load_2d(slot, mw, &c.full[s], kc, wrow);
+          if (NW == 2) ptx::tma_load_2d(slot + kChainTile * kChainTileK * 2, g.w1, &c.full[s], kc, wrow);
+          ptx::tma_load_2d(slot + NW * kChainTile * kChainTileK * 2, g.amap, &c.full[s], kc, 0);
+        }
+      }
+      DC_TRACE(0);
+      // ---------------- L2 prefetch of this CTA's unit in the next GEMM phase ----------------
+      if (ok && g.pf_tiles > 0) {
+        const int pn = g.pf_tiles * g.pf_nsplit;
+        for (int u = blockIdx.x; u < pn; u += gridDim.x) {
+          const int tile = u / g.pf_nsplit, split = u % g.pf_nsplit;
+          const int kb0 = (int)(((long long)split * g.pf_KB) / g.pf_nsplit);
+          int kb1 = (int)(((long long)(split + 1) * g.pf_KB) / g.pf_nsplit);
+          if (kb1 > kb0 + g.pf_kb) kb1 = kb0 + g.pf_kb;
+          const CUtensorMap* mw = g.pf_w0;
+          int wrow = tile * kChainTile;
+          bool both = g.pf_w1 != nullptr && g.pf_t1 == 0;  // gate and up: same rows of two maps
+          if (!both && g.pf_w2 != nullptr && tile >= g.pf_t2) { mw = g.pf_w2; wrow = (tile - g.pf_t2) * kChainTile; }
+          else if (!both && g.pf_w1 != nullptr && tile >= g.pf_t1) { mw = g.pf_w1; wrow = (tile - g.pf_t1) * kChainTile; }
+          for (int kb = kb0; kb < kb1; ++kb) {
+            ptx::tma_prefetch_l2_2d(mw, kb * kChainTileK, wrow);
+            if (both) ptx::tma_prefetch_l2_2d(g.pf_w1, kb * kChainTileK, wrow);
+          }
+        }
+      }
+    }
+  } else if (c.warp == 1) {
+    if (c.lane == 0) {
+      // ---------------- MMA issuer ----------------
+      const uint32_t idesc = ptx::idesc_bf16(kChainTile, BN);
+      bool ok = true;
+      int it = 0;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int split = u % g.nsplit;
+        const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
+        const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
+        if (c.units_done > 0) {  // the epilogue has drained both accumulators of the last unit
+          ok = ptx::mbar_wait(c.acc_empty, (c.units_done - 1) & 1u, c.abort_flag);
+          if (!ok) break;
+        }
+        ptx::tc_fence_after();
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % stages;
+          const uint32_t par = (c.use_bits >> s) & 1u;
+          c.use_bits ^= 1u << s;
+          ok = ptx::mbar_wait(&c.full[s], par, c.abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t slot = ptx::smem_u32(c.ring + (size_t)s * slot_bytes);
+          const uint64_t dw0 = ptx::smem_desc_sw128(slot);
+          const uint64_t dw1 = ptx::smem_desc_sw128(slot + kChainTile * kChainTileK * 2);
+          const uint64_t da = ptx::smem_desc_sw128(slot + NW * kChainTile * kChainTileK * 2);
+          const bool first = kb == kb0;
+#pragma unroll
+          for (int kk = 0; kk < kChainTileK / 16; ++kk) {
+            if (NW == 2) {
+              const uint32_t acc = (first && kk == 0) ? 0u : 1u;
+              ptx::umma_bf16(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
+              ptx::umma_bf16(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc, acc);
+            } else {
+              const uint32_t acc = (first && kk < 2) ? 0u : 1u;
+              ptx::umma_bf16(c.tmem_base + (kk & 1) * 256, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
+            }
+          }
+          ptx::umma_commit(&c.empty[s]);
+        }
+        if (ok) ptx::umma_commit(c.acc_full);
+        ++c.units_done;
+      }
+      DC_TRACE(1);
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+    const int quarter = c.warp & 3;
+    const int f = quarter * 32 + c.lane;  // feature inside the tile = TMEM lane
+    const uint32_t t_lane = c.tmem_base + ((uint32_t)(quarter * 32) << 16);
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      const int tile = u / g.nsplit, split = u % g.nsplit;
+      ok = ptx::mbar_wait(c.acc_full, c.units_done & 1u, c.abort_flag);
+      ++c.units_done;
+      if (!ok) break;
+      ptx::tc_fence_after();
+      // 16 columns (activation rows) at a time, in a rolled loop: the body stays small enough
+      // for the instruction cache (this code runs once per unit, so every miss is paid)
+      // 16 columns (activation rows) per step, two register buffers: the TMEM loads of the next
+      // step are in flight while this one is converted and stored.  BN equals M here (M is a
+      // multiple of 16), so every column is a real row.
+      float a0[16], a1[16], b0[16], b1[16];
+      ptx::tmem_ld_32x16(t_lane, a0);
+      ptx::tmem_ld_32x16(t_lane + 256, a1);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        ptx::tmem_ld_wait();
+        if (c0 + 16 < BN) {
+          ptx::tmem_ld_32x16(t_lane + c0 + 16, b0);
+          ptx::tmem_ld_32x16(t_lane + 256 + c0 + 16, b1);
+        }
+        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1);
+        if (c0 + 16 < BN) {
+          ptx::tmem_ld_wait();
+          if (c0 + 32 < BN) {
+            ptx::tmem_ld_32x16(t_lane + c0 + 32, a0);
+            ptx::tmem_ld_32x16(t_lane + 256 + c0 + 32, a1);
+          }
+          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1);
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(c.acc_empty);
+    }
+    if (threadIdx.x == 64) { DC_TRACE(2); }
+    // the outputs are read through TMA (async proxy) by other CTAs after the grid barrier
+    ptx::fence_proxy_async_all();
+    if (threadIdx.x == 64) { DC_TRACE(3); }
+  }
+}
+
+// x[row] += sum of the partial sums (in split order); out[row] = bf16(rmsnorm(x[row]) * g).
+// Two rows per CTA at a time: warps 0..2 take one, warps 3..5 the other.
+__device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, int nsplit,
+                                           const __nv_bfloat16* __restrict__ g, float* red) {
+  const int grp = c.warp / 3;                      // 0 or 1
+  const int t = threadIdx.x - grp * 96;            // 0..95 inside the group
+  const int d = p.d;
+  for (int r0 = 2 * blockIdx.x; r0 < p.M; r0 += 2 * gridDim.x) {
+    const int row = r0 + grp;
+    const bool live = row < p.M;
+    float ss = 0.f;
+    if (live) {
+      float* xr = p.x + (size_t)row * d;
+      const float* pr = p.part + (size_t)row * d;
+      for (int i = t * 4; i < d; i += 96 * 4) {
+        float4 v = *reinterpret_cast<const float4*>(xr + i);
+        if (nsplit > 0) {
+          for (int s = 0; s < nsplit; ++s) {
+            const float4 pv = __ldcg(reinterpret_cast<const float4*>(pr + (size_t)s * p.part_stride + i));
+            v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
+          }
+          *reinterpret_cast<float4*>(xr + i) = v;
+        }
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (c.lane == 0) red[c.warp] = ss;
+    // group-wide exchange: named barriers 2 and 3, 96 threads each
+    if (grp == 0) asm volatile("bar.sync 2, 96;" ::: "memory");
+    else asm volatile("bar.sync 3, 96;" ::: "memory");
+    const float tot = red[grp * 3] + red[grp * 3 + 1] + red[grp * 3 + 2];
+    if (live) {
+      const float inv = rsqrtf(tot / (float)d + p.eps);
+      const float* xr = p.x + (size_t)row * d;
+      __nv_bfloat16* outr = p.a + (size_t)row * d;
+      for (int i = t * 4; i < d; i += 96 * 4) {
+        const float4 v = *reinterpret_cast<const float4*>(xr + i);
+        const uint2 gw = *reinterpret_cast<const uint2*>(g + i);
+        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw.x);
+        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gw.y);
+        __nv_bfloat162 o01 = __floats2bfloat162_rn(v.x * inv * __low2float(g01), v.y * inv * __high2float(g01));
+        __nv_bfloat162 o23 = __floats2bfloat162_rn(v.z * inv * __low2float(g23), v.w * inv * __high2float(g23));
+        *reinterpret_cast<uint2*>(outr + i) =
+            make_uint2(*reinterpret_cast<uint32_t*>(&o01), *reinterpret_cast<uint32_t*>(&o23));
+      }
+    }
+    if (grp == 0) asm volatile("bar.sync 2, 96;" ::: "memory");
+    else asm volatile("bar.sync 3, 96;" ::: "memory");
+  }
+  ptx::fence_proxy_async_all();  // `a` is the next phase's TMA operand
+}
+
+__global__ void __launch_bounds__(kChainThreads, 1)
+k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc_full, bar_acc_empty;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+  __shared__ float red[8];
+
+  // an earlier kernel of this step gave up: leave everything alone (uniform over the grid, the
+  // word only changes inside a chain launch when one of its own waits expires)
+  if (*reinterpret_cast<volatile int32_t*>(p.status) != 0) return;
+
+  ChainCtx c;
+  c.ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                      ~static_cast<uintptr_t>(1023));
+  c.xch = reinterpret_cast<float*>(c.ring + kChainRing);
+  c.full = bar_full; c.empty = bar_empty; c.acc_full = &bar_acc_full; c.acc_empty = &bar_acc_empty;
+  c.abort_flag = &abort_flag;
+  c.fill_bits = 0; c.use_bits = 0; c.units_done = 0;
+  c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
+    ptx::mbar_init(&bar_acc_full, 1);
+    ptx::mbar_init(&bar_acc_empty, 128);
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&maps.wo); ptx::prefetch_tmap(&maps.wg); ptx::prefetch_tmap(&maps.wu);
+    ptx::prefetch_tmap(&maps.wd); ptx::prefetch_tmap(&maps.wq); ptx::prefetch_tmap(&maps.wk);
+    ptx::prefetch_tmap(&maps.wv); ptx::prefetch_tmap(&maps.a); ptx::prefetch_tmap(&maps.o);
+    ptx::prefetch_tmap(&maps.act);
+  }
+  if (c.warp == 1) {
+    ptx::tmem_alloc(&tmem_base_s, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  c.tmem_base = tmem_base_s;
+
+  const int KBd = p.d / kChainTileK, KBq = p.nq * 128 / kChainTileK, KBf = p.F / kChainTileK;
+  const int tiles_d = p.d / kChainTile, tiles_f = p.F / kChainTile, tiles_qkv = p.nq + 2 * p.nkv;
+  const bool has_qkv = p.phase_end > CH_QKV;
+
+  for (int ph = p.phase_begin; ph < p.phase_end; ++ph) {
+#ifdef DC_CHAIN_TRACE
+    if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph] = ptx::globaltimer();
+#endif
+    GemmPhase g{};
+    switch (ph) {
+      case CH_OPROJ:
+        g.w0 = &maps.wo; g.amap = &maps.o; g.tiles = tiles_d; g.nsplit = p.split_o; g.KB = KBq; g.N = p.d;
+        g.pf_w0 = &maps.wg; g.pf_w1 = &maps.wu; g.pf_t1 = 0; g.pf_tiles = tiles_f; g.pf_nsplit = 1;
+        g.pf_KB = KBd; g.pf_kb = 12;
+        chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
+        break;
+      case CH_NORM2:
+        chain_norm(c, p, p.split_o, p.g2, red);
+        break;
+      case CH_GATEUP:
+        g.w0 = &maps.wg; g.w1 = &maps.wu; g.amap = &maps.a; g.tiles = tiles_f; g.nsplit = 1; g.KB = KBd; g.N = p.F;
+        g.pf_w0 = &maps.wd; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_down; g.pf_KB = KBf; g.pf_kb = 16;
+        chain_gemm<CEPI_SWIGLU>(c, p, g, ph);
+        break;
+      case CH_DOWN:
+        g.w0 = &maps.wd; g.amap = &maps.act; g.tiles = tiles_d; g.nsplit = p.split_down; g.KB = KBf; g.N = p.d;
+        if (has_qkv) {
+          g.pf_w0 = &maps.wq; g.pf_w1 = &maps.wk; g.pf_w2 = &maps.wv; g.pf_t1 = p.nq; g.pf_t2 = p.nq + p.nkv;
+          g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = 16;
+        }
+        chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
+        break;
+      case CH_NORM1:
+        chain_norm(c, p, p.fold_norm1, p.g1, red);
+        break;
+      default:  // CH_QKV
+        g.w0 = &maps.wq; g.w1 = &maps.wk; g.w2 = &maps.wv; g.amap = &maps.a; g.tiles = tiles_qkv;
+        g.nsplit = 1; g.KB = KBd; g.N = 0;
+        // attention runs next; meanwhile the O projection of this layer streams into L2
+        g.pf_w0 = &maps.wo; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_o; g.pf_KB = KBq; g.pf_kb = 64;
+        chain_gemm<CEPI_QKV>(c, p, g, ph);
+        break;
+    }
+#ifdef DC_CHAIN_TRACE
+    __syncthreads();
+    if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph + 1] = ptx::globaltimer();
+#endif
+    if (ph + 1 < p.phase_end) {
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        if (abort_flag == 0 && !ptx::grid_barrier(p.bar, gridDim.x, p.status)) abort_flag = 1;
+        if (abort_flag) atomicExch(p.status, DC_ERR_TIMEOUT);
+        ptx::fence_proxy_async_all();
+      }
+      __syncthreads();
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (c.warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(c.tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && abort_flag) atomicExch(p.status, DC_ERR_TIMEOUT);
+#ifdef DC_CHAIN_TRACE
+  if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 12] = ptx::globaltimer();
+#endif
+}
+
+}  // namespace dc

@@ -81,6 +81,35 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return true;
 }
 
+// ---- grid-wide barrier for persistent kernels whose CTAs are all resident (cooperative launch) --
+// bar[0] counts arrivals, bar[1] is the generation.  The last arriver resets the count and bumps
+// the generation, so the words need no reset between launches.  One thread per CTA calls this
+// after a CTA-wide barrier.  The wait is bounded: returns false after kWaitLimitNs, or as soon as
+// *abort_word (global) is non-zero.
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n_ctas,
+                                             const int* abort_word) {
+  unsigned int gen, old;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(bar + 1) : "memory");
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(bar) : "memory");
+  if (old == n_ctas - 1) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], 0;" ::"l"(bar) : "memory");
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar + 1) : "memory");
+    return true;
+  }
+  const unsigned long long t0 = globaltimer();
+  unsigned int polls = 0;
+  while (true) {
+    unsigned int g;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(g) : "l"(bar + 1) : "memory");
+    if (g != gen) return true;
+    if ((++polls & 0x3f) == 0) {
+      int ab;
+      asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(ab) : "l"(abort_word) : "memory");
+      if (ab != 0 || globaltimer() - t0 > kWaitLimitNs) return false;
+    }
+  }
+}
+
 // ---- TMA: tiled 2-D / 3-D loads into shared memory, completion on an mbarrier -----------------
 // The innermost coordinate times the element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar,
@@ -106,6 +135,17 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       " [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
+}
+// Fire-and-forget prefetch of one box of a tiled tensor into L2 (no shared memory, no barrier).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+               ::"l"(map), "r"(c0), "r"(c1)
+               : "memory");
+}
+// Orders this thread's earlier generic-proxy writes (global or shared) before later async-proxy
+// (TMA) accesses, and the reverse.
+__device__ __forceinline__ void fence_proxy_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
