@@ -79,7 +79,7 @@ struct dc_ctx {
   float* tmp = nullptr;      // fp32 GEMM outputs of the CUDA-core path
   void* h = nullptr;         // LM-head input [M_lm, d]
   float* logits = nullptr;   // [M_lm, V] fp32, CUDA-core LM head only
-  float* cos_sin = nullptr;  // RoPE table [max_batch * R_cap_max, hd]
+  float* cos_sin = nullptr;  // RoPE table [max_batch * R_cap_max + 1, hd] (last row: angle step)
   int32_t* ws_pred = nullptr;
   float *ws_conf = nullptr, *ws_ent = nullptr, *ws_infl = nullptr, *ws_lse = nullptr;
   TcState* tc = nullptr;
@@ -421,7 +421,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
   c->x = ws_alloc<float>(c, M * g.d_model, &ok);
   c->a = ws_alloc<char>(c, M * g.d_model * es, &ok);
   c->h = ws_alloc<char>(c, (size_t)c->Mlm_max * g.d_model * es, &ok);
-  c->cos_sin = ws_alloc<float>(c, (size_t)g.max_batch * c->R_cap_max * hd, &ok);
+  c->cos_sin = ws_alloc<float>(c, ((size_t)g.max_batch * c->R_cap_max + 1) * hd, &ok);
   const size_t nw = (size_t)g.max_batch * g.max_window;
   c->ws_pred = ws_alloc<int32_t>(c, nw, &ok);
   c->ws_conf = ws_alloc<float>(c, nw, &ok);

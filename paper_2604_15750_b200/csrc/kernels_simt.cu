@@ -246,16 +246,18 @@ void launch_gemm_simt(const T* A, const T* W, float* C, int M, int N, int K, int
 
 // ---- RoPE ----------------------------------------------------------------------------------------
 // cos_sin[(b * R_cap + r) * hd + i] = cos(angle), [.. + hd/2 + i] = sin(angle),
-// angle = (ctx_len[b] + r) * theta^(-2i/hd), evaluated in double precision.
+// angle = (ctx_len[b] + r) * theta^(-2i/hd), evaluated in double precision.  Row batch * R_cap
+// holds cos / sin of theta^(-2i/hd) itself, the angle step between consecutive rows.
 __global__ void k_rope_table(SeqMeta m, int hd, float theta, float* __restrict__ cos_sin) {
   const int half = hd / 2;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  const int total = m.batch * m.R_cap * half;
+  const int rows = m.batch * m.R_cap;
+  const int total = (rows + 1) * half;   // one extra row: cos / sin of the per-row angle step
   if (idx >= total) return;
   const int i = idx % half, br = idx / half;
   const int r = br % m.R_cap, b = br / m.R_cap;
   const double inv_freq = pow((double)theta, -2.0 * (double)i / (double)hd);
-  const double ang = (double)(m.ctx_len[b] + r) * inv_freq;
+  const double ang = (br < rows) ? (double)(m.ctx_len[b] + r) * inv_freq : inv_freq;
   double sn, cs;
   sincos(ang, &sn, &cs);
   cos_sin[(size_t)br * hd + i] = (float)cs;
@@ -264,7 +266,7 @@ __global__ void k_rope_table(SeqMeta m, int hd, float theta, float* __restrict__
 
 void launch_rope_table(const SeqMeta& m, int head_dim, float theta, float* cos_sin,
                        cudaStream_t s) {
-  const int total = m.batch * m.R_cap * (head_dim / 2);
+  const int total = (m.batch * m.R_cap + 1) * (head_dim / 2);
   k_rope_table<<<(total + 255) / 256, 256, 0, s>>>(m, head_dim, theta, cos_sin);
 }
 

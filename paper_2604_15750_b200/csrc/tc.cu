@@ -319,9 +319,16 @@ int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k
 }
 
 bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
+  const dc_config& g = t->g;
   const int M = m.nv * m.batch * m.R_cap;
-  // one column block of at most 256 activation rows; the ring must hold two gate/up stages
-  return t->chain_grid > 0 && M <= 256;
+  // One column block of at most 256 activation rows.  The norm phases reuse the TMA ring as
+  // staging space, which needs at most one GEMM unit per CTA and phase, and both rows of a norm
+  // step (x plus the split-K partial sums) inside the ring.
+  const int units_qkv = g.n_q_heads + 2 * g.n_kv_heads, units_f = g.d_ff / kChainTile;
+  const int units_d = (g.d_model / kChainTile) * t->max_split;
+  const size_t norm_bytes = (size_t)2 * (1 + t->max_split) * g.d_model * sizeof(float) + g.d_model * 2;
+  return t->chain_grid > 0 && M <= 256 && units_qkv <= t->chain_grid && units_f <= t->chain_grid &&
+         units_d <= t->chain_grid && norm_bytes <= (size_t)kChainRing;
 }
 
 void tc_step_begin(TcState* t) {
@@ -379,7 +386,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
       cudaMemcpy(trace_buf, trace_dev, 256 * 64 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
       ++n_print;
       char fn[64];
-      snprintf(fn, sizeof(fn), "gpurun_out/chain_trace_dbg0_%d.txt", n_print);
+      snprintf(fn, sizeof(fn), "gpurun_out/chain_trace_dbg%s_%d.txt", getenv("DC_TAG") ? getenv("DC_TAG") : "0", n_print);
       FILE* f = fopen(fn, "w");
       if (f) {
         for (int c = 0; c < t->chain_grid; ++c) {

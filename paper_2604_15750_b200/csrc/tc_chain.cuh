@@ -54,7 +54,7 @@ struct ChainParams {
   const __nv_bfloat16* g2;      // norm2 gain of this layer
   const __nv_bfloat16* g1;      // norm1 gain of the layer phase 5 belongs to
   float eps;
-  const float* cos_sin;         // RoPE table [(b, r)][128]
+  const float* cos_sin;         // RoPE table [(b, r)][128]; row rows_per_variant: angle step
   int rows_per_variant;
   __nv_bfloat16 *q, *k, *v;     // q [M, nq*128], k [M, nkv*128], v transposed [nkv*128, ldv]
   int ldv;
@@ -71,17 +71,21 @@ constexpr int kChainXch = 128 * 17 * 4;         // RoPE exchange buffer of the Q
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
-constexpr int kPrefetchAhead = 8;              // k-blocks the L2 prefetch runs ahead of the TMA loads
+#ifndef DC_PREFETCH_AHEAD
+#define DC_PREFETCH_AHEAD 0
+#endif
+constexpr int kPrefetchAhead = DC_PREFETCH_AHEAD;              // k-blocks the L2 prefetch runs ahead of the TMA loads
 
 struct ChainCtx {
   uint8_t* ring;
   float* xch;
-  uint64_t *full, *empty, *acc_full, *acc_empty;
+  uint64_t *full, *empty, *acc_full, *acc_empty, *norm_bar;
   volatile int* abort_flag;
   uint32_t tmem_base;
   uint32_t fill_bits;   // producer: parity of the next fill of each slot
   uint32_t use_bits;    // MMA issuer: parity of the next use of each slot
   uint32_t units_done;  // accumulator hand-overs so far (MMA issuer and epilogue count alike)
+  uint32_t norm_uses;   // completed phases of norm_bar
   int warp, lane;
 };
 
@@ -101,11 +105,19 @@ struct GemmPhase {
 // Loads, MMAs and epilogue of one GEMM phase.  Every thread of the CTA calls it.
 enum { CEPI_PARTIAL = 0, CEPI_SWIGLU = 1, CEPI_QKV = 2 };
 
+// RoPE factors of one thread's feature pair index i: (cos, sin) of the first row of a chunk and
+// of the angle step between consecutive rows.  The rows of a chunk are consecutive positions, so
+// the factors of the following rows come from the rotation recurrence (16 steps in fp32: the
+// error stays far below a bf16 ulp).  This replaces 32 table reads per chunk, which sat on the
+// critical path behind the exchange barrier, by 2 reads issued one chunk ahead.
+struct RopeBase { float c, s, cd, sd; };
+
 // Epilogue of 16 accumulator columns (activation rows c0 .. c0+15) of feature f of a tile.
 template <int EPI>
 __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, const int N,
                                            const int tile, const int split, const int f,
-                                           const int c0, float (&v0)[16], float (&v1)[16]) {
+                                           const int c0, float (&v0)[16], float (&v1)[16],
+                                           const RopeBase rb) {
   if (EPI == CEPI_PARTIAL) {
     float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kChainTile + f) +
                  (size_t)c0 * N;
@@ -141,21 +153,20 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
 #pragma unroll
       for (int j = 0; j < 16; ++j) c.xch[f * 17 + j] = v0[j];
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      const int i = f & 63;
       const bool lo = f < 64;
       const bool is_k = tile >= p.nq;
       const int ld = is_k ? p.nkv * 128 : p.nq * 128;
       __nv_bfloat16* dst = (is_k ? p.k + (size_t)((tile - p.nq) * 128 + f)
                                  : p.q + (size_t)(tile * 128 + f)) + (size_t)c0 * ld;
-      int m0 = c0;  // a chunk of 16 rows never straddles the variants (rows_per_variant % 16 == 0)
-      if (m0 >= p.rows_per_variant) m0 -= p.rows_per_variant;  // prev variant: same table
-      const float* cs = p.cos_sin + (size_t)m0 * 128 + i;
+      float cv = rb.c, sv = rb.s;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float cv = __ldg(cs + j * 128), sv = __ldg(cs + j * 128 + 64);
         const float other = c.xch[(f ^ 64) * 17 + j];
         const float y = lo ? (v0[j] * cv - other * sv) : (v0[j] * cv + other * sv);
         dst[(size_t)j * ld] = __float2bfloat16_rn(y);
+        const float cn = cv * rb.cd - sv * rb.sd;
+        sv = sv * rb.cd + cv * rb.sd;
+        cv = cn;
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
@@ -202,9 +213,10 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           uint8_t* slot = c.ring + (size_t)s * slot_bytes;
           ptx::mbar_expect_tx(&c.full[s], (uint32_t)slot_bytes);
           const int kc = kb * kChainTileK;
-          // keep the HBM -> L2 stream kPrefetchAhead k-blocks ahead of the shared-memory ring:
-          // the ring alone (3..5 slots) cannot cover the HBM latency at full bandwidth
-          if (kb + kPrefetchAhead < kb1) {
+          // optional: keep an HBM -> L2 prefetch kPrefetchAhead k-blocks ahead of the ring.
+          // Measured slower than no prefetch at distances 4, 8 and 16 (the phases are bound by
+          // what an SM can take in from L2, not by HBM latency), so it is off by default.
+          if (kPrefetchAhead > 0 && kb + kPrefetchAhead < kb1) {
             ptx::tma_prefetch_l2_2d(mw, kc + kPrefetchAhead * kChainTileK, wrow);
             if (NW == 2) ptx::tma_prefetch_l2_2d(g.w1, kc + kPrefetchAhead * kChainTileK, wrow);
           }
@@ -287,15 +299,29 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
       const int tile = u / g.nsplit, split = u % g.nsplit;
+      // RoPE factors do not depend on the accumulators: fetch them while the MMAs still run
+      const bool rope = EPI == CEPI_QKV && tile < p.nq + p.nkv;
+      RopeBase rb{1.f, 0.f, 1.f, 0.f}, rb_next{1.f, 0.f, 1.f, 0.f};
+      auto rope_base = [&](int c0, RopeBase& r) {
+        int m0 = c0;  // a chunk of 16 rows never straddles the variants (rows_per_variant % 16 == 0)
+        if (m0 >= p.rows_per_variant) m0 -= p.rows_per_variant;  // prev variant: same table
+        const float* cs = p.cos_sin + (size_t)m0 * 128 + (f & 63);
+        r.c = __ldg(cs); r.s = __ldg(cs + 64);
+      };
+      if (rope) {
+        const float* dl = p.cos_sin + (size_t)p.rows_per_variant * 128 + (f & 63);  // step row
+        rb.cd = __ldg(dl); rb.sd = __ldg(dl + 64);
+        rb_next.cd = rb.cd; rb_next.sd = rb.sd;
+        rope_base(0, rb);
+      }
       ok = ptx::mbar_wait(c.acc_full, c.units_done & 1u, c.abort_flag);
       ++c.units_done;
       if (!ok) break;
       ptx::tc_fence_after();
-      // 16 columns (activation rows) at a time, in a rolled loop: the body stays small enough
-      // for the instruction cache (this code runs once per unit, so every miss is paid)
-      // 16 columns (activation rows) per step, two register buffers: the TMEM loads of the next
-      // step are in flight while this one is converted and stored.  BN equals M here (M is a
-      // multiple of 16), so every column is a real row.
+      // 16 columns (activation rows) per step in a rolled loop (the code runs once per unit, so
+      // it must stay small for the instruction cache), two register buffers: the TMEM loads of
+      // the next step are in flight while this one is converted and stored.  BN equals M here
+      // (M is a multiple of 16), so every column is a real row.
       float a0[16], a1[16], b0[16], b1[16];
       ptx::tmem_ld_32x16(t_lane, a0);
       ptx::tmem_ld_32x16(t_lane + 256, a1);
@@ -305,15 +331,17 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         if (c0 + 16 < BN) {
           ptx::tmem_ld_32x16(t_lane + c0 + 16, b0);
           ptx::tmem_ld_32x16(t_lane + 256 + c0 + 16, b1);
+          if (rope) rope_base(c0 + 16, rb_next);
         }
-        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1);
+        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb);
         if (c0 + 16 < BN) {
           ptx::tmem_ld_wait();
           if (c0 + 32 < BN) {
             ptx::tmem_ld_32x16(t_lane + c0 + 32, a0);
             ptx::tmem_ld_32x16(t_lane + 256 + c0 + 32, a1);
+            if (rope) rope_base(c0 + 32, rb);
           }
-          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1);
+          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1, rb_next);
         }
       }
       ptx::tc_fence_before();
@@ -327,27 +355,50 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
 }
 
 // x[row] += sum of the partial sums (in split order); out[row] = bf16(rmsnorm(x[row]) * g).
-// Two rows per CTA at a time: warps 0..2 take one, warps 3..5 the other.
+// Two rows per CTA at a time: warps 0..2 take one, warps 3..5 the other.  The rows of x and of
+// the partial sums are brought into the (idle) ring by bulk copies, so that a CTA has all of its
+// 160 KB in flight at once instead of a few loads per thread.
 __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, int nsplit,
-                                           const __nv_bfloat16* __restrict__ g, float* red) {
+                                           const __nv_bfloat16* __restrict__ g, float* red,
+                                           const int ph) {
   const int grp = c.warp / 3;                      // 0 or 1
   const int t = threadIdx.x - grp * 96;            // 0..95 inside the group
   const int d = p.d;
+  const int narr = 1 + nsplit;
+  float* stage = reinterpret_cast<float*>(c.ring);  // [grp][narr][d], then the gain vector
+  __nv_bfloat16* sg = reinterpret_cast<__nv_bfloat16*>(stage + (size_t)2 * narr * d);
   for (int r0 = 2 * blockIdx.x; r0 < p.M; r0 += 2 * gridDim.x) {
+    if (threadIdx.x == 0) {
+      const int rows = (r0 + 1 < p.M) ? 2 : 1;
+      ptx::fence_proxy_async_smem();  // earlier generic accesses to the staging space come first
+      ptx::mbar_expect_tx(c.norm_bar, (uint32_t)(rows * narr * d * 4 + d * 2));
+      ptx::bulk_load(sg, g, d * 2, c.norm_bar);
+      for (int gi = 0; gi < rows; ++gi) {
+        float* dst = stage + (size_t)gi * narr * d;
+        ptx::bulk_load(dst, p.x + (size_t)(r0 + gi) * d, d * 4, c.norm_bar);
+        for (int s = 0; s < nsplit; ++s)
+          ptx::bulk_load(dst + (size_t)(s + 1) * d,
+                         p.part + (size_t)s * p.part_stride + (size_t)(r0 + gi) * d, d * 4, c.norm_bar);
+      }
+    }
+    const bool got = ptx::mbar_wait(c.norm_bar, c.norm_uses & 1u, c.abort_flag);
+    ++c.norm_uses;
+    if (threadIdx.x == 0) { DC_TRACE(0); }
     const int row = r0 + grp;
-    const bool live = row < p.M;
+    const bool live = got && row < p.M;
+    float* sx = stage + (size_t)grp * narr * d;
     float ss = 0.f;
     if (live) {
       float* xr = p.x + (size_t)row * d;
-      const float* pr = p.part + (size_t)row * d;
       for (int i = t * 4; i < d; i += 96 * 4) {
-        float4 v = *reinterpret_cast<const float4*>(xr + i);
+        float4 v = *reinterpret_cast<const float4*>(sx + i);
         if (nsplit > 0) {
           for (int s = 0; s < nsplit; ++s) {
-            const float4 pv = __ldcg(reinterpret_cast<const float4*>(pr + (size_t)s * p.part_stride + i));
+            const float4 pv = *reinterpret_cast<const float4*>(sx + (size_t)(s + 1) * d + i);
             v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
           }
           *reinterpret_cast<float4*>(xr + i) = v;
+          *reinterpret_cast<float4*>(sx + i) = v;
         }
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
       }
@@ -355,17 +406,17 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (c.lane == 0) red[c.warp] = ss;
+    if (threadIdx.x == 0) { DC_TRACE(1); }
     // group-wide exchange: named barriers 2 and 3, 96 threads each
     if (grp == 0) asm volatile("bar.sync 2, 96;" ::: "memory");
     else asm volatile("bar.sync 3, 96;" ::: "memory");
     const float tot = red[grp * 3] + red[grp * 3 + 1] + red[grp * 3 + 2];
     if (live) {
       const float inv = rsqrtf(tot / (float)d + p.eps);
-      const float* xr = p.x + (size_t)row * d;
       __nv_bfloat16* outr = p.a + (size_t)row * d;
       for (int i = t * 4; i < d; i += 96 * 4) {
-        const float4 v = *reinterpret_cast<const float4*>(xr + i);
-        const uint2 gw = *reinterpret_cast<const uint2*>(g + i);
+        const float4 v = *reinterpret_cast<const float4*>(sx + i);
+        const uint2 gw = *reinterpret_cast<const uint2*>(sg + i);
         const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw.x);
         const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gw.y);
         __nv_bfloat162 o01 = __floats2bfloat162_rn(v.x * inv * __low2float(g01), v.y * inv * __high2float(g01));
@@ -374,8 +425,9 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
             make_uint2(*reinterpret_cast<uint32_t*>(&o01), *reinterpret_cast<uint32_t*>(&o23));
       }
     }
-    if (grp == 0) asm volatile("bar.sync 2, 96;" ::: "memory");
-    else asm volatile("bar.sync 3, 96;" ::: "memory");
+    // everyone is done with the staged rows before the next pair is loaded over them
+    __syncthreads();
+    if (threadIdx.x == 0) { DC_TRACE(2); }
   }
   ptx::fence_proxy_async_all();  // `a` is the next phase's TMA operand
 }
@@ -383,7 +435,7 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
 __global__ void __launch_bounds__(kChainThreads, 1)
 k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc_full, bar_acc_empty;
+  __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc_full, bar_acc_empty, bar_norm;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float red[8];
@@ -396,9 +448,9 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   c.ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                       ~static_cast<uintptr_t>(1023));
   c.xch = reinterpret_cast<float*>(c.ring + kChainRing);
-  c.full = bar_full; c.empty = bar_empty; c.acc_full = &bar_acc_full; c.acc_empty = &bar_acc_empty;
+  c.full = bar_full; c.empty = bar_empty; c.acc_full = &bar_acc_full; c.acc_empty = &bar_acc_empty; c.norm_bar = &bar_norm;
   c.abort_flag = &abort_flag;
-  c.fill_bits = 0; c.use_bits = 0; c.units_done = 0;
+  c.fill_bits = 0; c.use_bits = 0; c.units_done = 0; c.norm_uses = 0;
   c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -406,6 +458,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
     ptx::mbar_init(&bar_acc_full, 1);
     ptx::mbar_init(&bar_acc_empty, 128);
+    ptx::mbar_init(&bar_norm, 1);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&maps.wo); ptx::prefetch_tmap(&maps.wg); ptx::prefetch_tmap(&maps.wu);
     ptx::prefetch_tmap(&maps.wd); ptx::prefetch_tmap(&maps.wq); ptx::prefetch_tmap(&maps.wk);
@@ -438,7 +491,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
         break;
       case CH_NORM2:
-        chain_norm(c, p, p.split_o, p.g2, red);
+        chain_norm(c, p, p.split_o, p.g2, red, ph);
         break;
       case CH_GATEUP:
         g.w0 = &maps.wg; g.w1 = &maps.wu; g.amap = &maps.a; g.tiles = tiles_f; g.nsplit = 1; g.KB = KBd; g.N = p.F;
@@ -454,7 +507,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
         break;
       case CH_NORM1:
-        chain_norm(c, p, p.fold_norm1, p.g1, red);
+        chain_norm(c, p, p.fold_norm1, p.g1, red, ph);
         break;
       default:  // CH_QKV
         g.w0 = &maps.wq; g.w1 = &maps.wk; g.w2 = &maps.wv; g.amap = &maps.a; g.tiles = tiles_qkv;
