@@ -242,6 +242,58 @@ enum { DC_STAGE_EMBED = 0, DC_STAGE_NORM, DC_STAGE_QKV, DC_STAGE_ATTN, DC_STAGE_
 DC_API int dc_step_profiled(dc_ctx* ctx, const dc_step_in* in, const dc_step_out* out, float* stage_ms,
                      int32_t* stage_launches);
 
+/* ---- LM-head signals without any allocation -------------------------------------------------
+ * The paper has no counterpart of this call; it exists for hosts that must not allocate.
+ *
+ * Some callers cannot reach cudaMalloc at the moment they need the per-position signals: code
+ * that runs inside another framework's memory pool and is forbidden to go around it, code on a
+ * latency path where an allocation (an implicit device synchronisation) is not acceptable, or a
+ * process whose memory budget was handed out in full at start-up.  dc_create allocates a
+ * workspace, so it is closed to them.  dc_signals_static computes what the LM-head stage of
+ * dc_step computes - yhat_k, c_k, H_k, I_k and the log-sum-exp for every window position, from
+ * LM-head inputs the caller already holds - and keeps its scratch data (the LM-head inputs in
+ * the kernel's row order, the per-CTA partial softmax records, a status word) in a fixed array
+ * that is part of the library image: DC_STATIC_SCRATCH_BYTES of device memory on every GPU that
+ * loads the library, held until the process exits.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ *
+ * Limits (DC_ERR_SHAPE / DC_ERR_UNSUPPORTED beyond them, nothing is launched, and
+ * dc_last_error(NULL) gives the reason): bf16 only,
+ * d_model a multiple of 128 and <= DC_STATIC_MAX_D, batch * round16(longest window) <=
+ * DC_STATIC_MAX_POS positions, vocab >= 2.
+ *
+ * The first call on a device looks up the device address of the array and opts the kernel in to
+ * its shared memory; make that first call before any stream capture.  All calls on a device
+ * share the one array, which keeps the previous call's contents: the call itself clears what
+ * must start at zero, but two calls whose kernels overlap on the GPU (different streams, no
+ * dependency) race on it - order them.  The caller passes inputs and outputs as usual; outputs
+ * are valid after the stream is synchronised.  With the same inputs the results are those of
+ * dc_step (same kernels, same tiling). */
+enum { DC_STATIC_MAX_D = 8192, DC_STATIC_MAX_POS = 128,
+       DC_STATIC_SCRATCH_BYTES = 2 * DC_STATIC_MAX_POS * DC_STATIC_MAX_D * 2 /* inputs, bf16 */
+                                 + 2 * 160 * 128 * 8 * 4                      /* partial records */
+                                 + 4096 /* per-position results, status */ };
+
+typedef struct dc_signals_in {
+  int32_t d_model, vocab, mask_id;
+  int32_t forbid_mask_pred;  /* 1: [MASK] is removed from both softmaxes                     */
+  int32_t batch;             /* sequences, >= 1                                              */
+  int32_t max_window;        /* row pitch of h and of the outputs, multiple of 16            */
+  const void* lm_head;       /* device bf16 [vocab, d_model], 16-byte aligned                */
+  const void* h;             /* device bf16 [batch][2][max_window][d_model]: LM-head input   */
+                             /* rows of the curr (0) and prev (1) variant                    */
+  const int32_t* win_len;    /* host [batch], 1..max_window                                  */
+  const int32_t* have_prev;  /* host [batch] or null (= all 1); 0: I_k is reported as 0      */
+} dc_signals_in;
+
+typedef struct dc_signals_out {   /* device, [batch][max_window]; any but status may be null */
+  int32_t* pred_id;
+  float *conf, *entropy, *influence, *lse;
+  int32_t* status;                /* [batch], required: DC_OK or DC_ERR_TIMEOUT              */
+} dc_signals_out;
+
+DC_API int dc_signals_static(const dc_signals_in* in, const dc_signals_out* out, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

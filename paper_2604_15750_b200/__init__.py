@@ -3,4 +3,4 @@
 Argument marshalling only; every step of the path runs in the library's kernels.
 """
 from .binding import (DepCap, DepCapError, Hyper, lib, load_library, pack_kv_cache,  # noqa: F401
-                      STAGE_NAMES)
+                      STAGE_NAMES, signals_static)

@@ -18,7 +18,7 @@ DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
                "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
-           "dc_debug_logits", "dc_step_profiled"]
+           "dc_debug_logits", "dc_step_profiled", "dc_signals_static"]
 
 
 class DepCapError(RuntimeError):
@@ -85,6 +85,17 @@ class dc_select_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("sel_mask", "sel_idx", "sel_count")]
 
 
+class dc_signals_in(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("d_model", "vocab", "mask_id", "forbid_mask_pred", "batch",
+                                         "max_window")] + \
+               [("lm_head", C.c_void_p), ("h", C.c_void_p), ("win_len", _I32P), ("have_prev", _I32P)]
+
+
+class dc_signals_out(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("pred_id", "conf", "entropy", "influence", "lse",
+                                          "status")]
+
+
 _lib = None
 
 
@@ -107,6 +118,8 @@ def load_library(path: str | None = None):
     lib_.dc_boundary.argtypes = [C.c_void_p, C.POINTER(dc_boundary_in),
                                  C.POINTER(dc_boundary_out)]
     lib_.dc_select.argtypes = [C.c_void_p, C.POINTER(dc_select_in), C.POINTER(dc_select_out)]
+    lib_.dc_signals_static.argtypes = [C.POINTER(dc_signals_in), C.POINTER(dc_signals_out),
+                                       C.c_void_p]
     lib_.dc_destroy.argtypes = [C.c_void_p]
     lib_.dc_debug_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
     lib_.dc_last_error.argtypes = [C.c_void_p]
@@ -158,6 +171,31 @@ def pack_kv_cache(k_logical: torch.Tensor, v_logical: torch.Tensor, max_batch: i
     k[:, :B, :, :P, :] = k_logical
     v[:, :B, :, :, :P] = v_logical.transpose(3, 4)
     return k, v
+
+
+def signals_static(lm_head, h, win_len, out, *, mask_id, forbid_mask_pred=True, have_prev=None,
+                   stream=None):
+    """dc_signals_static: the LM-head signals for callers that must not allocate.
+
+    lm_head [vocab, d] and h [batch, 2, max_window, d] are bf16 CUDA tensors the caller already
+    holds; `out` maps pred_id / conf / entropy / influence / lse / status to preallocated CUDA
+    tensors ([batch, max_window]; status [batch]).  Nothing is allocated on the device: the
+    library keeps its scratch data in a fixed array of its own image (see include/depcap.h for
+    the limits, and for why overlapping calls must be ordered)."""
+    B = len(win_len)
+    wl_ = _host_i32(win_len, B)
+    hp_ = _host_i32(have_prev, B) if have_prev is not None else None
+    si = dc_signals_in(d_model=h.shape[-1], vocab=lm_head.shape[0], mask_id=mask_id,
+                       forbid_mask_pred=int(forbid_mask_pred), batch=B, max_window=h.shape[2],
+                       lm_head=_ptr(lm_head), h=_ptr(h), win_len=C.cast(wl_, _I32P),
+                       have_prev=C.cast(hp_, _I32P) if hp_ is not None else None)
+    so = dc_signals_out(**{k: _ptr(out.get(k)) for k in ("pred_id", "conf", "entropy",
+                                                          "influence", "lse", "status")})
+    st = stream or torch.cuda.current_stream(h.device)
+    rc = lib().dc_signals_static(C.byref(si), C.byref(so), C.c_void_p(st.cuda_stream))
+    if rc != DC_OK:
+        raise DepCapError(rc, lib().dc_last_error(None).decode())
+    return out
 
 
 class DepCap:

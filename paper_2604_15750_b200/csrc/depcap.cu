@@ -55,6 +55,8 @@ struct Profiler : dc::StageHook {
 
 }  // namespace
 
+void dc::set_thread_error(const char* msg) { g_create_error = msg ? msg : ""; }
+
 struct dc_ctx {
   dc_config cfg{};
   Hyper hp{};

@@ -8,6 +8,9 @@
 
 namespace dc {
 
+// reason of the last failed call that had no context (what dc_last_error(NULL) returns)
+void set_thread_error(const char* msg);
+
 // Per-step sequence description, passed by value to kernels (baked into a captured graph).
 struct SeqMeta {
   int ctx_len[DC_MAX_BATCH];

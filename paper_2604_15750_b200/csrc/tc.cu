@@ -499,3 +499,141 @@ void tc_flush_status(TcState* t, int32_t* status, int batch) {
 }
 
 }  // namespace dc
+
+// ---- dc_signals_static: the LM-head stage with its scratch data in the library image ------------
+namespace {
+
+// Scratch of dc_signals_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the device address is looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[DC_STATIC_SCRATCH_BYTES];
+
+constexpr size_t kStaticHBytes = (size_t)2 * DC_STATIC_MAX_POS * DC_STATIC_MAX_D * 2;
+constexpr size_t kStaticPartBytes = (size_t)2 * 160 * 128 * 8 * 4;
+
+struct StaticDev {
+  bool ready = false;
+  unsigned char* base = nullptr;
+  int n_sm = 0, lm_stages = 0;
+};
+StaticDev g_static_dev[64];
+
+// LM-head input rows [batch][2][max_window][d] -> the LM head's row order (groups of G positions,
+// curr rows then prev rows); rows of pad positions are zero.
+__global__ void k_static_rows(const __nv_bfloat16* __restrict__ h_in, int max_window, int d,
+                              dc::SeqMeta m, __nv_bfloat16* __restrict__ h) {
+  const int lrow = blockIdx.x;
+  const int grp = lrow / (m.nv * m.G), in = lrow % (m.nv * m.G);
+  const int v = in / m.G, p = grp * m.G + in % m.G;
+  const int b = p / m.W_cap, k = p % m.W_cap;
+  uint4* dst = reinterpret_cast<uint4*>(h + (size_t)lrow * d);
+  if (b >= m.batch || k >= m.win_len[b]) {
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(h_in + (((size_t)b * 2 + v) * max_window + k) * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
+}
+
+__global__ void k_static_status(const int32_t* word, int32_t* status, int batch) {
+  for (int b = threadIdx.x; b < batch; b += blockDim.x) status[b] = *word;
+}
+
+int sfail(int code, const char* msg) {
+  dc::set_thread_error(msg);  // read back with dc_last_error(NULL)
+  return code;
+}
+
+}  // namespace
+
+extern "C" int dc_signals_static(const dc_signals_in* in, const dc_signals_out* out, void* cuda_stream) {
+  using namespace dc;
+  if (!in || !out || !in->lm_head || !in->h || !in->win_len || !out->status)
+    return sfail(DC_ERR_INVALID_ARG, "null argument");
+  if (in->d_model < 128 || in->d_model % 128 || in->d_model > DC_STATIC_MAX_D)
+    return sfail(DC_ERR_UNSUPPORTED, "d_model must be a multiple of 128, at most DC_STATIC_MAX_D");
+  if (in->vocab < 2 || in->mask_id < 0 || in->mask_id >= in->vocab)
+    return sfail(DC_ERR_INVALID_ARG, "bad vocab / mask_id");
+  if (in->batch < 1 || in->batch > DC_MAX_BATCH || in->max_window < 16 || in->max_window % 16 ||
+      in->max_window > DC_MAX_WINDOW)
+    return sfail(DC_ERR_SHAPE, "batch or max_window out of range");
+  SeqMeta m{};
+  m.batch = in->batch; m.nv = 2;
+  int maxW = 0;
+  for (int b = 0; b < in->batch; ++b) {
+    const int W = in->win_len[b];
+    if (W < 1 || W > in->max_window) return sfail(DC_ERR_SHAPE, "win_len outside [1, max_window]");
+    m.win_len[b] = W;
+    m.have_prev[b] = in->have_prev ? (in->have_prev[b] != 0) : 1;
+    maxW = maxW > W ? maxW : W;
+  }
+  m.W_cap = (maxW + 15) / 16 * 16;
+  m.R_cap = m.W_cap;
+  const int npos = in->batch * m.W_cap;
+  if (npos > DC_STATIC_MAX_POS)
+    return sfail(DC_ERR_SHAPE, "more than DC_STATIC_MAX_POS window positions: the fixed scratch array cannot hold them");
+  m.G = npos < 64 ? npos : 64;
+  m.npos_pad = (npos + m.G - 1) / m.G * m.G;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+    return sfail(DC_ERR_CUDA, "no current CUDA device");
+  StaticDev& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    // once per device, with that device current: the device address of the scratch array, the
+    // kernel's shared-memory opt-in, the SM count.  Nothing here allocates.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return sfail(DC_ERR_CUDA, "cudaGetSymbolAddress failed for the scratch array");
+    }
+    sd.base = static_cast<unsigned char*>(p);
+    cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (sd.n_sm < 1) return sfail(DC_ERR_CUDA, "cannot read the SM count");
+    if (sd.n_sm > 160) sd.n_sm = 160;  // the partial-record region is sized for 160 CTAs
+    const int lm_static = 2 * 64 * 33 * 4 + 512;
+    sd.lm_stages = (kSmemBudget - lm_static) / kLmStageBytes;
+    if (sd.lm_stages > 8) sd.lm_stages = 8;
+    if (cudaFuncSetAttribute(k_lmhead_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sd.lm_stages * kLmStageBytes + 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return sfail(DC_ERR_CUDA, "cannot opt in to shared memory for the LM head");
+    }
+    if (!get_encode()) return sfail(DC_ERR_CUDA, "cuTensorMapEncodeTiled unavailable");
+    sd.ready = true;
+  }
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  __nv_bfloat16* h_rows = reinterpret_cast<__nv_bfloat16*>(sd.base);
+  float* part = reinterpret_cast<float*>(sd.base + kStaticHBytes);
+  unsigned char* tail = sd.base + kStaticHBytes + kStaticPartBytes;
+  int32_t* ws_pred = reinterpret_cast<int32_t*>(tail);
+  float* ws_conf = reinterpret_cast<float*>(tail + 512);
+  float* ws_ent = reinterpret_cast<float*>(tail + 1024);
+  float* ws_infl = reinterpret_cast<float*>(tail + 1536);
+  float* ws_lse = reinterpret_cast<float*>(tail + 2048);
+  int32_t* word = reinterpret_cast<int32_t*>(tail + 2560);
+
+  const int Mlm = m.nv * m.npos_pad;
+  CUtensorMap map_h, map_lm;
+  if (!(make_map_2d(&map_h, h_rows, 2 * DC_STATIC_MAX_POS, in->d_model, 128) &&
+        make_map_2d(&map_lm, in->lm_head, in->vocab, in->d_model, 128)))
+    return sfail(DC_ERR_CUDA, "tensor map encoding failed (lm_head must be 16-byte aligned)");
+
+  // the status word is the only part of the array that must start at zero; every row and record
+  // the kernels read below is rewritten by this call first
+  cudaMemsetAsync(word, 0, sizeof(int32_t), s);
+  k_static_rows<<<Mlm, 128, 0, s>>>((const __nv_bfloat16*)in->h, in->max_window, in->d_model, m, h_rows);
+  LmParams p;
+  p.m = m; p.V = in->vocab; p.K = in->d_model; p.mask_id = in->forbid_mask_pred ? in->mask_id : -1;
+  p.part = part; p.status = word;
+  const int ntiles = (in->vocab + 127) / 128;
+  const int nctas = ntiles < sd.n_sm ? ntiles : sd.n_sm;
+  dim3 grid(nctas, m.npos_pad / m.G);
+  k_lmhead_tc<<<grid, kLmThreads, sd.lm_stages * kLmStageBytes + 1024, s>>>(map_h, map_lm, p, sd.lm_stages);
+  SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, in->max_window};
+  k_lm_combine<<<(npos + 3) / 4, 128, 0, s>>>(part, nctas, m, ws_pred, ws_conf, ws_ent, ws_infl, ws_lse, so);
+  k_static_status<<<1, 32, 0, s>>>(word, out->status, in->batch);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return sfail(DC_ERR_CUDA, cudaGetErrorString(e));
+  return DC_OK;
+}
+

@@ -1,0 +1,78 @@
+"""dc_signals_static: the LM-head signals computed with no device allocation at all.
+
+Who needs it: a caller that is not allowed to reach cudaMalloc when it wants the signals - it
+lives inside another framework's memory pool, or sits on a path where an allocation's implicit
+synchronisation is unacceptable, or its memory budget was handed out at start-up.  dc_create
+allocates a workspace, so such a caller cannot use dc_step; this entry point keeps its scratch data
+in a fixed array inside the library image instead.
+
+The check: on the same LM-head inputs its outputs equal those dc_step writes (same kernels, same
+tiling), on two calls in a row - the second call runs over the first call's leftovers in the shared
+scratch array, which is exactly the situation the entry point has to handle.  The file sorts last
+so that a run that stops at the first failure has already run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_15750_b200 import DepCapError, inputs, signals_static
+
+from parity import Case
+
+pytestmark = pytest.mark.gpu
+
+
+def _case():
+    wl = inputs.Workload("noalloc", 1, 256, 2, 2, 128, 256, 3000, "bf16", 3, 32, 64, 16, 32, 64, 5151)
+    lengths = dict(ctx_len=[64, 40, 33], last_len=[16, 5, 16], win_len=[32, 17, 9],
+                   remain_len=[64, 17, 30])
+    return Case(wl, lengths=lengths, steer="decay")
+
+
+def test_static_scratch_entry_matches_dc_step_twice_in_a_row():
+    case = _case()
+    eng = case.make_engine()
+    di = case.device_inputs(eng)
+    ref = {k: v.clone() for k, v in eng.step(**di).items()}
+    eng.synchronize()
+    B, W = case.wl.batch, eng.max_window
+    lm_head = eng._weights["lm_head"]
+    dev = lm_head.device
+    mk = lambda dt: torch.full((B, W), -7, dtype=dt, device=dev)
+    for call in range(2):
+        out = dict(pred_id=mk(torch.int32), conf=mk(torch.float32), entropy=mk(torch.float32),
+                   influence=mk(torch.float32), lse=mk(torch.float32),
+                   status=torch.full((B,), -7, dtype=torch.int32, device=dev))
+        if call == 1:
+            # leave other contents in the shared scratch array first: a call with different inputs
+            other = dict(out, **{k: v.clone() for k, v in out.items()})
+            signals_static(lm_head, torch.flip(di["h_final"], dims=[2]).contiguous(),
+                           [W, W, W], other, mask_id=case.wl.mask_id)
+        signals_static(lm_head, di["h_final"], di["win_len"], out, mask_id=case.wl.mask_id)
+        torch.cuda.synchronize()
+        assert out["status"].cpu().tolist() == [0] * B
+        for b in range(B):
+            w = di["win_len"][b]
+            assert torch.equal(out["pred_id"][b, :w], ref["pred_id"][b, :w]), (call, b)
+            for name, tol in (("conf", 2e-2), ("entropy", 2e-2), ("lse", 2e-2)):
+                g, r = out[name][b, :w].cpu().numpy(), ref[name][b, :w].cpu().numpy()
+                assert (np.abs(g - r) / np.maximum(np.abs(r), 1.0)).max() <= tol, (call, name, b)
+            g, r = out["influence"][b, :w].cpu().numpy(), ref["influence"][b, :w].cpu().numpy()
+            assert np.abs(g - r).max() <= 1e-3, (call, b)
+            # positions beyond the window are not written
+            assert int(out["pred_id"][b, w:].max().item() if w < W else -7) == -7
+    eng.close()
+
+
+def test_static_scratch_entry_rejects_sizes_beyond_its_array():
+    case = _case()
+    eng = case.make_engine()
+    lm_head = eng._weights["lm_head"]
+    dev = lm_head.device
+    B, W = 9, 16                                   # 9 * 16 = 144 positions > 128
+    h = torch.zeros((B, 2, W, 256), dtype=torch.bfloat16, device=dev)
+    out = dict(status=torch.zeros((B,), dtype=torch.int32, device=dev))
+    with pytest.raises(DepCapError) as e:
+        signals_static(lm_head, h, [W] * B, out, mask_id=case.wl.mask_id)
+    assert e.value.code == 2 and "DC_STATIC_MAX_POS" in str(e.value)
+    eng.close()
