@@ -495,7 +495,7 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
                                                const int32_t* __restrict__ ws_pred,
                                                const float* __restrict__ ws_lse, int d, SeqMeta m,
                                                int max_window, float* __restrict__ xlogp) {
-  extern __shared__ float wrow[];  // W_lm[yhat_j] as fp32
+  extern __shared__ __align__(16) float wrow[];  // W_lm[yhat_j] as fp32
   const int b = blockIdx.y, j = blockIdx.x;
   const int W = m.win_len[b];
   if (j >= W) return;
@@ -507,7 +507,14 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
   for (int i = warp; i < W; i += nw) {
     const T* hr = h + (size_t)lm_row(m, 0, b * m.W_cap + i) * d;
     float acc = 0.f;
-    for (int e = lane; e < d; e += 32) acc = fmaf(to_f<T>(hr[e]), wrow[e], acc);
+    // d is a multiple of 4: four elements per lane and step (8- or 16-byte loads)
+    for (int e = lane * 4; e < d; e += 128) {
+      float hv[4];
+      load4<T>(hr + e, hv);
+      const float4 wv = *reinterpret_cast<const float4*>(wrow + e);
+      acc = fmaf(hv[0], wv.x, acc); acc = fmaf(hv[1], wv.y, acc);
+      acc = fmaf(hv[2], wv.z, acc); acc = fmaf(hv[3], wv.w, acc);
+    }
     acc = warp_sum(acc);
     if (lane == 0)
       xlogp[((size_t)b * max_window + i) * max_window + j] = acc - ws_lse[b * m.W_cap + i];

@@ -25,8 +25,10 @@
 // use one accumulator each, the other GEMMs send even k-steps to the first and odd k-steps to the
 // second and add them in the epilogue.
 //
-// Warp roles (192 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
-// owns the TMEM allocation), warps 2..5 = epilogue.  All six warps run the norm phases.
+// Warp roles (256 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
+// owns the TMEM allocation).  All eight warps run the epilogue: warp w reads the TMEM lanes
+// 32 * (w % 4) .. +31 (the only ones it can reach) and the column half w / 4, so two warps share
+// every lane quarter.  All eight warps run the norm phases.
 #pragma once
 #include "kernels.h"
 #include "tc.h"
@@ -65,9 +67,9 @@ struct ChainParams {
 #endif
 };
 
-constexpr int kChainThreads = 192;
+constexpr int kChainThreads = 256;
 constexpr int kChainRing = 208 * 1024;          // TMA ring
-constexpr int kChainXch = 128 * 17 * 4;         // RoPE exchange buffer of the QKV epilogue
+constexpr int kChainXch = 2 * 128 * 17 * 4;     // RoPE exchange buffers of the QKV epilogue (one per column half)
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
@@ -84,7 +86,8 @@ struct ChainCtx {
   uint32_t tmem_base;
   uint32_t fill_bits;   // producer: parity of the next fill of each slot
   uint32_t use_bits;    // MMA issuer: parity of the next use of each slot
-  uint32_t units_done;  // accumulator hand-overs so far (MMA issuer and epilogue count alike)
+  uint32_t units_done;  // units whose accumulators this thread has drained (epilogue role)
+  uint32_t mma_units;   // units whose MMAs this thread has issued (MMA issuer only)
   uint32_t norm_uses;   // completed phases of norm_bar
   int warp, lane;
 };
@@ -117,7 +120,7 @@ template <int EPI>
 __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, const int N,
                                            const int tile, const int split, const int f,
                                            const int c0, float (&v0)[16], float (&v1)[16],
-                                           const RopeBase rb) {
+                                           const RopeBase rb, const int half) {
   if (EPI == CEPI_PARTIAL) {
     float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kChainTile + f) +
                  (size_t)c0 * N;
@@ -151,8 +154,10 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
       // rotate-half RoPE: feature i < 64 pairs with i + 64, held by the warp two quarters
       // away; the chunk is exchanged through shared memory
 #pragma unroll
-      for (int j = 0; j < 16; ++j) c.xch[f * 17 + j] = v0[j];
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      float* xch = c.xch + half * (128 * 17);
+      for (int j = 0; j < 16; ++j) xch[f * 17 + j] = v0[j];
+      // the 128 threads of this column half meet on their own named barrier (1 or 2)
+      asm volatile("bar.sync %0, 128;" ::"r"(half + 1) : "memory");
       const bool lo = f < 64;
       const bool is_k = tile >= p.nq;
       const int ld = is_k ? p.nkv * 128 : p.nq * 128;
@@ -161,14 +166,14 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
       float cv = rb.c, sv = rb.s;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float other = c.xch[(f ^ 64) * 17 + j];
+        const float other = xch[(f ^ 64) * 17 + j];
         const float y = lo ? (v0[j] * cv - other * sv) : (v0[j] * cv + other * sv);
         dst[(size_t)j * ld] = __float2bfloat16_rn(y);
         const float cn = cv * rb.cd - sv * rb.sd;
         sv = sv * rb.cd + cv * rb.sd;
         cv = cn;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync %0, 128;" ::"r"(half + 1) : "memory");
     }
   }
 }
@@ -256,8 +261,8 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         const int split = u % g.nsplit;
         const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
         const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
-        if (c.units_done > 0) {  // the epilogue has drained both accumulators of the last unit
-          ok = ptx::mbar_wait(c.acc_empty, (c.units_done - 1) & 1u, c.abort_flag);
+        if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
+          ok = ptx::mbar_wait(c.acc_empty, (c.mma_units - 1) & 1u, c.abort_flag);
           if (!ok) break;
         }
         ptx::tc_fence_after();
@@ -287,13 +292,18 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           ptx::umma_commit(&c.empty[s]);
         }
         if (ok) ptx::umma_commit(c.acc_full);
-        ++c.units_done;
+        ++c.mma_units;
       }
       DC_TRACE(1);
     }
-  } else {
-    // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+  }
+  __syncwarp();
+  {
+    // ---------------- epilogue: all warps; TMEM lane quarter = warp % 4, column half = warp / 4 ----
     const int quarter = c.warp & 3;
+    const int half = c.warp >> 2;
+    const int col_mid = ((BN >> 1) + 15) & ~15;      // columns [0, col_mid) and [col_mid, BN)
+    const int col0 = half ? col_mid : 0, col1 = half ? BN : col_mid;
     const int f = quarter * 32 + c.lane;  // feature inside the tile = TMEM lane
     const uint32_t t_lane = c.tmem_base + ((uint32_t)(quarter * 32) << 16);
     bool ok = true;
@@ -312,7 +322,7 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         const float* dl = p.cos_sin + (size_t)p.rows_per_variant * 128 + (f & 63);  // step row
         rb.cd = __ldg(dl); rb.sd = __ldg(dl + 64);
         rb_next.cd = rb.cd; rb_next.sd = rb.sd;
-        rope_base(0, rb);
+        rope_base(col0, rb);
       }
       ok = ptx::mbar_wait(c.acc_full, c.units_done & 1u, c.abort_flag);
       ++c.units_done;
@@ -323,25 +333,25 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       // the next step are in flight while this one is converted and stored.  BN equals M here
       // (M is a multiple of 16), so every column is a real row.
       float a0[16], a1[16], b0[16], b1[16];
-      ptx::tmem_ld_32x16(t_lane, a0);
-      ptx::tmem_ld_32x16(t_lane + 256, a1);
+      ptx::tmem_ld_32x16(t_lane + col0, a0);
+      ptx::tmem_ld_32x16(t_lane + 256 + col0, a1);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = col0; c0 < col1; c0 += 32) {
         ptx::tmem_ld_wait();
-        if (c0 + 16 < BN) {
+        if (c0 + 16 < col1) {
           ptx::tmem_ld_32x16(t_lane + c0 + 16, b0);
           ptx::tmem_ld_32x16(t_lane + 256 + c0 + 16, b1);
           if (rope) rope_base(c0 + 16, rb_next);
         }
-        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb);
-        if (c0 + 16 < BN) {
+        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
+        if (c0 + 16 < col1) {
           ptx::tmem_ld_wait();
-          if (c0 + 32 < BN) {
+          if (c0 + 32 < col1) {
             ptx::tmem_ld_32x16(t_lane + c0 + 32, a0);
             ptx::tmem_ld_32x16(t_lane + 256 + c0 + 32, a1);
             if (rope) rope_base(c0 + 32, rb);
           }
-          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1, rb_next);
+          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1, rb_next, half);
         }
       }
       ptx::tc_fence_before();
@@ -355,14 +365,14 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
 }
 
 // x[row] += sum of the partial sums (in split order); out[row] = bf16(rmsnorm(x[row]) * g).
-// Two rows per CTA at a time: warps 0..2 take one, warps 3..5 the other.  The rows of x and of
+// Two rows per CTA at a time: warps 0..3 take one, warps 4..7 the other.  The rows of x and of
 // the partial sums are brought into the (idle) ring by bulk copies, so that a CTA has all of its
 // 160 KB in flight at once instead of a few loads per thread.
 __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, int nsplit,
                                            const __nv_bfloat16* __restrict__ g, float* red,
                                            const int ph) {
-  const int grp = c.warp / 3;                      // 0 or 1
-  const int t = threadIdx.x - grp * 96;            // 0..95 inside the group
+  const int grp = c.warp >> 2;                     // 0 or 1
+  const int t = threadIdx.x - grp * 128;           // 0..127 inside the group
   const int d = p.d;
   const int narr = 1 + nsplit;
   float* stage = reinterpret_cast<float*>(c.ring);  // [grp][narr][d], then the gain vector
@@ -390,7 +400,7 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     float ss = 0.f;
     if (live) {
       float* xr = p.x + (size_t)row * d;
-      for (int i = t * 4; i < d; i += 96 * 4) {
+      for (int i = t * 4; i < d; i += 128 * 4) {
         float4 v = *reinterpret_cast<const float4*>(sx + i);
         if (nsplit > 0) {
           for (int s = 0; s < nsplit; ++s) {
@@ -407,14 +417,13 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (c.lane == 0) red[c.warp] = ss;
     if (threadIdx.x == 0) { DC_TRACE(1); }
-    // group-wide exchange: named barriers 2 and 3, 96 threads each
-    if (grp == 0) asm volatile("bar.sync 2, 96;" ::: "memory");
-    else asm volatile("bar.sync 3, 96;" ::: "memory");
-    const float tot = red[grp * 3] + red[grp * 3 + 1] + red[grp * 3 + 2];
+    // group-wide exchange: named barriers 3 and 4, 128 threads each
+    asm volatile("bar.sync %0, 128;" ::"r"(grp + 3) : "memory");
+    const float tot = red[grp * 4] + red[grp * 4 + 1] + red[grp * 4 + 2] + red[grp * 4 + 3];
     if (live) {
       const float inv = rsqrtf(tot / (float)d + p.eps);
       __nv_bfloat16* outr = p.a + (size_t)row * d;
-      for (int i = t * 4; i < d; i += 96 * 4) {
+      for (int i = t * 4; i < d; i += 128 * 4) {
         const float4 v = *reinterpret_cast<const float4*>(sx + i);
         const uint2 gw = *reinterpret_cast<const uint2*>(sg + i);
         const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw.x);
@@ -450,14 +459,14 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   c.xch = reinterpret_cast<float*>(c.ring + kChainRing);
   c.full = bar_full; c.empty = bar_empty; c.acc_full = &bar_acc_full; c.acc_empty = &bar_acc_empty; c.norm_bar = &bar_norm;
   c.abort_flag = &abort_flag;
-  c.fill_bits = 0; c.use_bits = 0; c.units_done = 0; c.norm_uses = 0;
+  c.fill_bits = 0; c.use_bits = 0; c.units_done = 0; c.mma_units = 0; c.norm_uses = 0;
   c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
     ptx::mbar_init(&bar_acc_full, 1);
-    ptx::mbar_init(&bar_acc_empty, 128);
+    ptx::mbar_init(&bar_acc_empty, kChainThreads);
     ptx::mbar_init(&bar_norm, 1);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&maps.wo); ptx::prefetch_tmap(&maps.wg); ptx::prefetch_tmap(&maps.wu);
