@@ -507,8 +507,21 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
   for (int i = warp; i < W; i += nw) {
     const T* hr = h + (size_t)lm_row(m, 0, b * m.W_cap + i) * d;
     float acc = 0.f;
-    // d is a multiple of 4: four elements per lane and step (8- or 16-byte loads)
-    for (int e = lane * 4; e < d; e += 128) {
+    // d is a multiple of 4: four elements per lane and step (8- or 16-byte loads), eight steps
+    // in flight at a time (the loop is bound by the latency of the h loads otherwise)
+    int e = lane * 4;
+    for (; e + 7 * 128 < d; e += 8 * 128) {
+      float hv[8][4];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) load4<T>(hr + e + u * 128, hv[u]);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float4 wv = *reinterpret_cast<const float4*>(wrow + e + u * 128);
+        acc = fmaf(hv[u][0], wv.x, acc); acc = fmaf(hv[u][1], wv.y, acc);
+        acc = fmaf(hv[u][2], wv.z, acc); acc = fmaf(hv[u][3], wv.w, acc);
+      }
+    }
+    for (; e < d; e += 128) {
       float hv[4];
       load4<T>(hr + e, hv);
       const float4 wv = *reinterpret_cast<const float4*>(wrow + e);

@@ -99,6 +99,7 @@ struct TcState {
   int n_sm = 148, lm_stages = 6;
   unsigned int* grid_bar = nullptr;  // {count, generation} of the dense chain's grid barrier
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
+  bool chain_coop = false;           // launched cooperatively (co-residency guaranteed)
   std::string err;
   bool attrs_set = false;
 };
@@ -233,16 +234,26 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
     t->grid_bar = talloc<unsigned int>(t, 2, &ok);
     if (!ok) return tfail(t, DC_ERR_NOMEM, "dense-chain workspace allocation failed");
     cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), s);
-    int dev = 0, coop = 0, per_sm = 0;
+    int dev = 0, coop = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (coop &&
-        cudaFuncSetAttribute(k_dense_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem) ==
-            cudaSuccess &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_dense_chain, kChainThreads, kChainSmem) ==
-            cudaSuccess &&
-        per_sm >= 1)
-      t->chain_grid = t->n_sm;
+    if (cudaFuncSetAttribute(k_dense_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem) ==
+        cudaSuccess) {
+      // one CTA per SM in clusters of two: all of them must be resident at once
+      cudaLaunchConfig_t cfg{};
+      const int grid = t->n_sm & ~1;
+      cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kChainThreads); cfg.dynamicSmemBytes = kChainSmem;
+      cudaLaunchAttribute attr;
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+      cfg.attrs = &attr; cfg.numAttrs = 1;
+      int n_clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, k_dense_chain, &cfg) == cudaSuccess &&
+          2 * n_clusters >= grid && grid >= 2) {
+        t->chain_grid = grid;
+        t->chain_coop = coop != 0;
+      }
+    }
     cudaGetLastError();
   }
   return DC_OK;
@@ -327,7 +338,9 @@ bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
   const int units_qkv = g.n_q_heads + 2 * g.n_kv_heads, units_f = g.d_ff / kChainTile;
   const int units_d = (g.d_model / kChainTile) * t->max_split;
   const size_t norm_bytes = (size_t)2 * (1 + t->max_split) * g.d_model * sizeof(float) + g.d_model * 2;
-  return t->chain_grid > 0 && M <= 256 && units_qkv <= t->chain_grid && units_f <= t->chain_grid &&
+  const bool even = g.n_q_heads % 2 == 0 && g.n_kv_heads % 2 == 0 && (g.d_model / kChainTile) % 2 == 0 &&
+                    (g.d_ff / kChainTile) % 2 == 0;   // a CTA pair takes two adjacent tiles of one matrix
+  return t->chain_grid > 0 && even && M >= 32 && M <= 256 && units_qkv <= t->chain_grid && units_f <= t->chain_grid &&
          units_d <= t->chain_grid && norm_bytes <= (size_t)kChainRing;
 }
 
@@ -345,7 +358,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   const int M = m.nv * m.batch * m.R_cap;
   const int BN = (M + 15) / 16 * 16;
   ActMaps* am = nullptr;
-  int rc = get_act_maps(t, a, BN, &am);
+  int rc = get_act_maps(t, a, BN / 2, &am);  // every CTA of a pair stages half of the rows
   if (rc != DC_OK) return rc;
   ChainMaps maps;
   const LayerMaps& L = t->layers[layer];
@@ -375,9 +388,16 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   cudaMemsetAsync(trace_dev, 0, 256 * 64 * sizeof(unsigned long long), t->s);
   p.trace = trace_dev;
 #endif
-  void* args[] = {&maps, &p};
-  cudaError_t e = cudaLaunchCooperativeKernel((const void*)k_dense_chain, dim3(t->chain_grid),
-                                              dim3(kChainThreads), args, kChainSmem, t->s);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(t->chain_grid); cfg.blockDim = dim3(kChainThreads);
+  cfg.dynamicSmemBytes = kChainSmem; cfg.stream = t->s;
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeClusterDimension;
+  attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+  attrs[1].id = cudaLaunchAttributeCooperative;
+  attrs[1].val.cooperative = 1;
+  cfg.attrs = attrs; cfg.numAttrs = t->chain_coop ? 2 : 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_dense_chain, maps, p);
 #ifdef DC_CHAIN_TRACE
   {
     static int n_print = 0;

@@ -25,6 +25,14 @@
 // use one accumulator each, the other GEMMs send even k-steps to the first and odd k-steps to the
 // second and add them in the epilogue.
 //
+// CTA pairs: the launch uses clusters of two CTAs and every MMA is a pair MMA (cta_group::2,
+// M = 256): each CTA streams its own 128 weight rows but only HALF of the activation rows, the
+// tensor cores of both SMs read the two halves from both shared memories.  What an SM can take in
+// from L2 (about 100 GB/s, measured) bounds these GEMMs, and the activation tile is the part of
+// that traffic that carries no new information; halving it is worth 15..30% per phase.  The even
+// CTA of a pair issues the MMAs; TMA loads of both CTAs report to the even CTA's full barrier,
+// tcgen05.commit releases the ring slot in both CTAs.  No load is multicast.
+//
 // Warp roles (256 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
 // owns the TMEM allocation).  All eight warps run the epilogue: warp w reads the TMEM lanes
 // 32 * (w % 4) .. +31 (the only ones it can reach) and the column half w / 4, so two warps share
@@ -39,7 +47,7 @@ namespace dc {
 struct ChainMaps {
   CUtensorMap wo, wg, wu, wd;   // this layer: [d, hq], [F, d], [F, d], [d, F]
   CUtensorMap wq, wk, wv;       // the layer whose QKV phase 5 computes
-  CUtensorMap a, o, act;        // activation operands, box = BN rows x 64 columns
+  CUtensorMap a, o, act;        // activation operands, box = BN/2 rows x 64 columns (one CTA's half)
 };
 
 struct ChainParams {
@@ -76,6 +84,17 @@ constexpr int kChainTileK = 64;
 #ifndef DC_PREFETCH_AHEAD
 #define DC_PREFETCH_AHEAD 0
 #endif
+#ifndef DC_PF_GU
+#define DC_PF_GU 4
+#endif
+#ifndef DC_PF_DN
+#define DC_PF_DN 4
+#endif
+#ifndef DC_PF_QKV
+#define DC_PF_QKV 4
+#endif
+// k-blocks of its next unit that a CTA prefetches into L2 when its own loads are issued
+constexpr int kPfGateUp = DC_PF_GU, kPfDown = DC_PF_DN, kPfQkv = DC_PF_QKV;
 constexpr int kPrefetchAhead = DC_PREFETCH_AHEAD;              // k-blocks the L2 prefetch runs ahead of the TMA loads
 
 struct ChainCtx {
@@ -90,6 +109,7 @@ struct ChainCtx {
   uint32_t mma_units;   // units whose MMAs this thread has issued (MMA issuer only)
   uint32_t norm_uses;   // completed phases of norm_bar
   int warp, lane;
+  uint32_t rank;        // 0 / 1 inside the CTA pair
 };
 
 struct GemmPhase {
@@ -105,7 +125,14 @@ struct GemmPhase {
   int pf_tiles, pf_nsplit, pf_KB, pf_kb, pf_t1, pf_t2;  // pf_t1 / pf_t2: first tile of w1 / w2
 };
 
-// Loads, MMAs and epilogue of one GEMM phase.  Every thread of the CTA calls it.
+// CTA-level unit u -> (weight tile, K split).  CTAs 2p and 2p+1 form a pair and must hold adjacent
+// tiles of the same split: pair unit u / 2 = tile_pair * nsplit + split.
+__device__ __forceinline__ void chain_unit(int u, int nsplit, int& tile, int& split) {
+  const int pp = u >> 1;
+  tile = (pp / nsplit) * 2 + (u & 1);
+  split = pp % nsplit;
+}
+
 enum { CEPI_PARTIAL = 0, CEPI_SWIGLU = 1, CEPI_QKV = 2 };
 
 // RoPE factors of one thread's feature pair index i: (cos, sin) of the first row of a chunk and
@@ -189,7 +216,8 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
                                            const int ph) {
   constexpr int NW = (EPI == CEPI_SWIGLU) ? 2 : 1;
   const int BN = p.BN;
-  const int slot_bytes = NW * kChainTile * kChainTileK * 2 + BN * kChainTileK * 2;
+  const int half_rows = BN >> 1;  // activation rows this CTA stages (the pair MMA reads both halves)
+  const int slot_bytes = NW * kChainTile * kChainTileK * 2 + half_rows * kChainTileK * 2;
   int stages = kChainRing / slot_bytes;
   if (stages > 8) stages = 8;
   const int n_units = g.tiles * g.nsplit;
@@ -198,9 +226,14 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
     if (c.lane == 0) {
       // ---------------- TMA producer ----------------
       bool ok = true;
-      int it = 0;
+      const uint32_t ring0 = ptx::smem_u32(c.ring);
+      const uint32_t full0 = ptx::smem_u32(&c.full[0]), empty0 = ptx::smem_u32(&c.empty[0]);
+      const uint32_t full_remote0 = c.rank == 0 ? full0 : ptx::mapa_shared(full0, 0);
+      const int arow = (int)c.rank * half_rows;
+      uint32_t ps = 0, pslot = ring0;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const int tile = u / g.nsplit, split = u % g.nsplit;
+        int tile, split;
+        chain_unit(u, g.nsplit, tile, split);
         const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
         const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
         const CUtensorMap* mw = g.w0;
@@ -209,25 +242,31 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           if (tile >= p.nq + p.nkv) { mw = g.w2; wrow = (tile - p.nq - p.nkv) * kChainTile; }
           else if (tile >= p.nq) { mw = g.w1; wrow = (tile - p.nq) * kChainTile; }
         }
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % stages;
-          const uint32_t par = (c.fill_bits >> s) & 1u;
-          c.fill_bits ^= 1u << s;
-          ok = ptx::mbar_wait(&c.empty[s], par ^ 1u, c.abort_flag);
+        // lean loop: slot index, addresses and coordinates advance by additions only
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const uint32_t par = (c.fill_bits >> ps) & 1u;
+          c.fill_bits ^= 1u << ps;
+#ifdef DC_CHAIN_TRACE
+          const long long tw0 = clock64();
+#endif
+          ok = ptx::mbar_wait_a(empty0 + 8u * ps, par ^ 1u, c.abort_flag);
+#ifdef DC_CHAIN_TRACE
+          p.trace[blockIdx.x * 64 + 41 + ph * 4] += (unsigned long long)(clock64() - tw0);
+#endif
           if (!ok) break;
-          uint8_t* slot = c.ring + (size_t)s * slot_bytes;
-          ptx::mbar_expect_tx(&c.full[s], (uint32_t)slot_bytes);
+          // the bytes of both CTAs are credited to the even CTA's barrier, which its MMA issuer
+          // waits on
+          if (c.rank == 0) ptx::mbar_expect_tx_a(full0 + 8u * ps, 2u * (uint32_t)slot_bytes);
+          const uint32_t bar = full_remote0 + 8u * ps;
           const int kc = kb * kChainTileK;
-          // optional: keep an HBM -> L2 prefetch kPrefetchAhead k-blocks ahead of the ring.
-          // Measured slower than no prefetch at distances 4, 8 and 16 (the phases are bound by
-          // what an SM can take in from L2, not by HBM latency), so it is off by default.
           if (kPrefetchAhead > 0 && kb + kPrefetchAhead < kb1) {
             ptx::tma_prefetch_l2_2d(mw, kc + kPrefetchAhead * kChainTileK, wrow);
             if (NW == 2) ptx::tma_prefetch_l2_2d(g.w1, kc + kPrefetchAhead * kChainTileK, wrow);
           }
-          ptx::tma_load_2d(slot, mw, &c.full[s], kc, wrow);
-          if (NW == 2) ptx::tma_load_2d(slot + kChainTile * kChainTileK * 2, g.w1, &c.full[s], kc, wrow);
-          ptx::tma_load_2d(slot + NW * kChainTile * kChainTileK * 2, g.amap, &c.full[s], kc, 0);
+          ptx::tma_load_2d_pair_a(pslot, mw, bar, kc, wrow);
+          if (NW == 2) ptx::tma_load_2d_pair_a(pslot + kChainTile * kChainTileK * 2, g.w1, bar, kc, wrow);
+          ptx::tma_load_2d_pair_a(pslot + NW * kChainTile * kChainTileK * 2, g.amap, bar, kc, arow);
+          if (++ps == (uint32_t)stages) { ps = 0; pslot = ring0; } else pslot += (uint32_t)slot_bytes;
         }
       }
       DC_TRACE(0);
@@ -235,7 +274,8 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       if (ok && g.pf_tiles > 0) {
         const int pn = g.pf_tiles * g.pf_nsplit;
         for (int u = blockIdx.x; u < pn; u += gridDim.x) {
-          const int tile = u / g.pf_nsplit, split = u % g.pf_nsplit;
+          int tile, split;
+          chain_unit(u, g.pf_nsplit, tile, split);
           const int kb0 = (int)(((long long)split * g.pf_KB) / g.pf_nsplit);
           int kb1 = (int)(((long long)(split + 1) * g.pf_KB) / g.pf_nsplit);
           if (kb1 > kb0 + g.pf_kb) kb1 = kb0 + g.pf_kb;
@@ -252,13 +292,17 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       }
     }
   } else if (c.warp == 1) {
-    if (c.lane == 0) {
-      // ---------------- MMA issuer ----------------
-      const uint32_t idesc = ptx::idesc_bf16(kChainTile, BN);
+    if (c.lane == 0 && c.rank == 0) {
+      // ---------------- MMA issuer (even CTA of the pair, for both) ----------------
+      const uint32_t idesc = ptx::idesc_bf16(2 * kChainTile, BN);
       bool ok = true;
-      int it = 0;
+      const uint32_t mring0 = ptx::smem_u32(c.ring);
+      const uint32_t mfull0 = ptx::smem_u32(&c.full[0]), mempty0 = ptx::smem_u32(&c.empty[0]);
+      const uint64_t desc_hi = ptx::smem_desc_sw128_hi();
+      uint32_t ms = 0, mslot = mring0;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const int split = u % g.nsplit;
+        int tile, split;
+        chain_unit(u, g.nsplit, tile, split);
         const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
         const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
         if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
@@ -266,32 +310,46 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           if (!ok) break;
         }
         ptx::tc_fence_after();
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % stages;
-          const uint32_t par = (c.use_bits >> s) & 1u;
-          c.use_bits ^= 1u << s;
-          ok = ptx::mbar_wait(&c.full[s], par, c.abort_flag);
+        uint32_t acc_first = 0;   // 0 until the first k-block of the unit has been issued
+#ifdef DC_CHAIN_TRACE
+        const long long tl0 = clock64();
+#endif
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const uint32_t par = (c.use_bits >> ms) & 1u;
+          c.use_bits ^= 1u << ms;
+#ifdef DC_CHAIN_TRACE
+          const long long tw0 = clock64();
+#endif
+          ok = ptx::mbar_wait_a(mfull0 + 8u * ms, par, c.abort_flag);
+#ifdef DC_CHAIN_TRACE
+          p.trace[blockIdx.x * 64 + 40 + ph * 4] += (unsigned long long)(clock64() - tw0);
+#endif
           if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t slot = ptx::smem_u32(c.ring + (size_t)s * slot_bytes);
-          const uint64_t dw0 = ptx::smem_desc_sw128(slot);
-          const uint64_t dw1 = ptx::smem_desc_sw128(slot + kChainTile * kChainTileK * 2);
-          const uint64_t da = ptx::smem_desc_sw128(slot + NW * kChainTile * kChainTileK * 2);
-          const bool first = kb == kb0;
+          const uint64_t dw0 = desc_hi | (uint64_t)(mslot >> 4);
+          const uint64_t dw1 = dw0 + (kChainTile * kChainTileK * 2 >> 4);
+          const uint64_t da = dw0 + (NW * kChainTile * kChainTileK * 2 >> 4);
+          if (NW == 2) {
+            ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+            ptx::umma_bf16_pair(c.tmem_base + 256, dw1, da, idesc, acc_first);
 #pragma unroll
-          for (int kk = 0; kk < kChainTileK / 16; ++kk) {
-            if (NW == 2) {
-              const uint32_t acc = (first && kk == 0) ? 0u : 1u;
-              ptx::umma_bf16(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
-              ptx::umma_bf16(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc, acc);
-            } else {
-              const uint32_t acc = (first && kk < 2) ? 0u : 1u;
-              ptx::umma_bf16(c.tmem_base + (kk & 1) * 256, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
+            for (int kk = 1; kk < kChainTileK / 16; ++kk) {
+              ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
+              ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
             }
+          } else {
+            ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+            ptx::umma_bf16_pair(c.tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
+            ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 4, da + 4, idesc);
+            ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw0 + 6, da + 6, idesc);
           }
-          ptx::umma_commit(&c.empty[s]);
+          acc_first = 1;
+          ptx::umma_commit_pair_a(mempty0 + 8u * ms);   // frees the slot in both CTAs
+          if (++ms == (uint32_t)stages) { ms = 0; mslot = mring0; } else mslot += (uint32_t)slot_bytes;
         }
-        if (ok) ptx::umma_commit(c.acc_full);
+#ifdef DC_CHAIN_TRACE
+        p.trace[blockIdx.x * 64 + 42 + ph * 4] += (unsigned long long)(clock64() - tl0);
+#endif
+        if (ok) ptx::umma_commit_pair(c.acc_full);  // both epilogues start
         ++c.mma_units;
       }
       DC_TRACE(1);
@@ -308,7 +366,8 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
     const uint32_t t_lane = c.tmem_base + ((uint32_t)(quarter * 32) << 16);
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const int tile = u / g.nsplit, split = u % g.nsplit;
+      int tile, split;
+      chain_unit(u, g.nsplit, tile, split);
       // RoPE factors do not depend on the accumulators: fetch them while the MMAs still run
       const bool rope = EPI == CEPI_QKV && tile < p.nq + p.nkv;
       RopeBase rb{1.f, 0.f, 1.f, 0.f}, rb_next{1.f, 0.f, 1.f, 0.f};
@@ -449,10 +508,6 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   __shared__ int abort_flag;
   __shared__ float red[8];
 
-  // an earlier kernel of this step gave up: leave everything alone (uniform over the grid, the
-  // word only changes inside a chain launch when one of its own waits expires)
-  if (*reinterpret_cast<volatile int32_t*>(p.status) != 0) return;
-
   ChainCtx c;
   c.ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                       ~static_cast<uintptr_t>(1023));
@@ -461,9 +516,12 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   c.abort_flag = &abort_flag;
   c.fill_bits = 0; c.use_bits = 0; c.units_done = 0; c.mma_units = 0; c.norm_uses = 0;
   c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
+  c.rank = ptx::cluster_ctarank();
 
   if (threadIdx.x == 0) {
-    abort_flag = 0;
+    // an earlier kernel of this step gave up: run through without touching anything (every CTA
+    // still reaches the cluster barriers below)
+    abort_flag = (*reinterpret_cast<volatile int32_t*>(p.status) != 0) ? 1 : 0;
     for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
     ptx::mbar_init(&bar_acc_full, 1);
     ptx::mbar_init(&bar_acc_empty, kChainThreads);
@@ -482,6 +540,11 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   __syncthreads();
   ptx::tc_fence_after();
   c.tmem_base = tmem_base_s;
+  // both CTAs of a pair hold all 512 columns, so the pair MMA's accumulator address (the even
+  // CTA's) names the same columns in the odd CTA; anything else would be a silent mix-up
+  if (threadIdx.x == 0 && c.tmem_base != 0) abort_flag = 1;
+  // the partner's barriers are initialised before any of its loads can report to them
+  ptx::cluster_sync();
 
   const int KBd = p.d / kChainTileK, KBq = p.nq * 128 / kChainTileK, KBf = p.F / kChainTileK;
   const int tiles_d = p.d / kChainTile, tiles_f = p.F / kChainTile, tiles_qkv = p.nq + 2 * p.nkv;
@@ -492,11 +555,12 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph] = ptx::globaltimer();
 #endif
     GemmPhase g{};
-    switch (ph) {
+    const bool dead = abort_flag != 0;   // uniform: written before the last CTA-wide barrier
+    if (!dead) switch (ph) {
       case CH_OPROJ:
         g.w0 = &maps.wo; g.amap = &maps.o; g.tiles = tiles_d; g.nsplit = p.split_o; g.KB = KBq; g.N = p.d;
         g.pf_w0 = &maps.wg; g.pf_w1 = &maps.wu; g.pf_t1 = 0; g.pf_tiles = tiles_f; g.pf_nsplit = 1;
-        g.pf_KB = KBd; g.pf_kb = 12;
+        g.pf_KB = KBd; g.pf_kb = kPfGateUp;
         chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
         break;
       case CH_NORM2:
@@ -504,14 +568,14 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         break;
       case CH_GATEUP:
         g.w0 = &maps.wg; g.w1 = &maps.wu; g.amap = &maps.a; g.tiles = tiles_f; g.nsplit = 1; g.KB = KBd; g.N = p.F;
-        g.pf_w0 = &maps.wd; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_down; g.pf_KB = KBf; g.pf_kb = 16;
+        g.pf_w0 = &maps.wd; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_down; g.pf_KB = KBf; g.pf_kb = kPfDown;
         chain_gemm<CEPI_SWIGLU>(c, p, g, ph);
         break;
       case CH_DOWN:
         g.w0 = &maps.wd; g.amap = &maps.act; g.tiles = tiles_d; g.nsplit = p.split_down; g.KB = KBf; g.N = p.d;
         if (has_qkv) {
           g.pf_w0 = &maps.wq; g.pf_w1 = &maps.wk; g.pf_w2 = &maps.wv; g.pf_t1 = p.nq; g.pf_t2 = p.nq + p.nkv;
-          g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = 16;
+          g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = kPfQkv;
         }
         chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
         break;
@@ -543,6 +607,9 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
 
   ptx::tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair leaves while the other may still read its shared memory or signal its
+  // barriers
+  ptx::cluster_sync();
   if (c.warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(c.tmem_base, 512);
