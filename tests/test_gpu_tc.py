@@ -76,3 +76,19 @@ def test_tc_more_than_128_active_rows_and_long_context():
     gpu, ora = case.run_gpu(eng, poison=True), case.run_oracle()
     compare(case, gpu, ora)
     eng.close()
+
+
+def test_fused_dense_chain_is_the_path_taken_when_the_rows_fit_one_block():
+    """M = 2 * 2 * 48 = 192 activation rows: the persistent dense chain must run (one launch that
+    starts the step plus one per layer), not the per-op kernels; with 3 * 48 * 2 = 288 rows the
+    per-op kernels run."""
+    for batch, fused in ((2, True), (3, False)):
+        case = Case(_wl(batch))
+        eng = case.make_engine()
+        di = case.device_inputs(eng)
+        _, launches = eng.step_profiled(**di)
+        if fused:
+            assert launches["dense"] == case.n_layers + 1 and launches["qkv"] == 0
+        else:
+            assert launches["dense"] == 0 and launches["qkv"] == case.n_layers
+        eng.close()
