@@ -26,7 +26,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2604_15750_b200 import inputs  # noqa: E402
+from paper_2604_15750_b200 import inputs, replicas  # noqa: E402
 
 METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"
@@ -222,7 +222,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     n_layers = args.layers or wl.n_layers
     # each replica draws its own sequences (seed offset by rank); weights are the same model
-    wl_r = inputs.scaled(wl, seed=wl.seed + 1000 * rank) if rank else wl
+    wl_r = inputs.scaled(wl, seed=replicas.replica_seed(wl.seed, rank)) if rank else wl
     weights, k_log, v_log, toks, lens, steer = _setup(wl, dev, n_layers)
     if rank:
         toks = inputs.make_tokens(wl_r)
@@ -312,13 +312,8 @@ def main():
 
     # ---- reduce over ranks --------------------------------------------------------------------
     ms_step = ms_total / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_step, e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, e2e_ms = float(t[0]), float(t[1])
-        cnt = torch.tensor([committed, committed_e2e], device=dev, dtype=torch.int64)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        committed, committed_e2e = int(cnt[0]), int(cnt[1])
+    (ms_step, e2e_ms), (committed, committed_e2e) = replicas.combine(
+        dist, [ms_step, e2e_ms], [committed, committed_e2e], device=dev)
     if rank != 0:
         eng.close()
         if dist is not None:
