@@ -242,6 +242,25 @@ __device__ __forceinline__ void tma_load_2d_pair_a(uint32_t dst, const CUtensorM
       " [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1) : "memory");
 }
+// L2 eviction policies for TMA loads: weights are read once per step (evict first), the small
+// activation / partial-sum buffers are re-read by every CTA (evict last)
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar_addr,
+                                                      int c0, int c1, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void umma_commit_pair_a(uint32_t bar) {
   const uint16_t mask = 3;
   asm volatile(
