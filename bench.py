@@ -93,10 +93,12 @@ class ClockSampler:
         return out
 
 
-def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=16):
+def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=16, budget_s=None):
     """Times the CPU oracle, as it stands, on a bounded sample of the step for sequence 0:
-    one transformer layer (curr and prev variants) and the LM head + signals on the first
-    n_head_pos window positions; the full-step time is extrapolated from the two."""
+    one transformer layer (curr and prev variants) over the first n_rows active rows and the LM
+    head + signals on the first n_head_pos window positions; the full-step time is extrapolated
+    (the layer cost is linear in the rows, the head cost in the positions).  budget_s shrinks the
+    sample so that one call takes about that long (a full sample is about 5 s)."""
     import numpy as np
     from oracle import adapters
     from oracle import depcap_oracle as O
@@ -105,6 +107,12 @@ def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=
     ow = adapters.weights_from_torch(one)
     ocfg = adapters.config_from_workload(wl, n_layers=1)
     P, Lb, W = lens["ctx_len"][0], lens["last_len"][0], lens["win_len"][0]
+    R = Lb + W
+    n_rows = R
+    if budget_s is not None:
+        frac = min(1.0, budget_s / 5.0)
+        n_rows = max(4, min(R, int(R * frac)))
+        n_head_pos = max(2, min(n_head_pos, int(n_head_pos * frac)))
     kc = adapters.to_np(k_log[:1, 0]) if k_log is not None else None
     vc = adapters.to_np(v_log[:1, 0]) if v_log is not None else None
     last = toks["last_ids"][0, :Lb].numpy()
@@ -112,11 +120,11 @@ def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=
     tok_curr = np.concatenate([last, win]).astype(np.int64)
     tok_prev = tok_curr.copy(); tok_prev[:Lb] = wl.mask_id
     t0 = time.perf_counter()
-    O.forward(ocfg, ow, tok_curr, P, kc[:, :, :P] if kc is not None else None,
+    O.forward(ocfg, ow, tok_curr[:n_rows], P, kc[:, :, :P] if kc is not None else None,
               vc[:, :, :P] if vc is not None else None, n_layers=1)
-    O.forward(ocfg, ow, tok_prev, P, kc[:, :, :P] if kc is not None else None,
+    O.forward(ocfg, ow, tok_prev[:n_rows], P, kc[:, :, :P] if kc is not None else None,
               vc[:, :, :P] if vc is not None else None, n_layers=1)
-    t_layer = time.perf_counter() - t0
+    t_layer = (time.perf_counter() - t0) * (R / n_rows)
     n = min(n_head_pos, W)
     hf = (adapters.to_np(steer[0, 0, :n]), adapters.to_np(steer[0, 1, :n]))
     t0 = time.perf_counter()
@@ -124,9 +132,9 @@ def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=
     t_head = time.perf_counter() - t0
     est = wl.n_layers * t_layer + t_head * (W / n)
     return dict(t_layer=t_layer, t_head=t_head, est_step_s=est * wl.batch,
-                sample=f"sequence 0: 1 of {wl.n_layers} layers (curr+prev variants) + LM head/"
-                       f"signals/decisions on {n} of {W} window positions; extrapolated to "
-                       f"{wl.n_layers} layers, {W} positions, batch {wl.batch}")
+                sample=f"sequence 0: 1 of {wl.n_layers} layers (curr+prev variants) on {n_rows} of {R} "
+                       f"active rows + LM head/signals/decisions on {n} of {W} window positions; "
+                       f"extrapolated to {wl.n_layers} layers, {R} rows, {W} positions, batch {wl.batch}")
 
 
 def _oracle_committed(wl, weights_dev, toks, lens, steer):
@@ -146,6 +154,15 @@ def _oracle_committed(wl, weights_dev, toks, lens, steer):
                    toks["win_ids"][b, :W].numpy(), lens["remain_len"][b], h_final=hf)
         total += len(o["selected"])
     return total
+
+
+def _config(wl, n_layers, **extra):
+    """The workload description both arms print."""
+    c = dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
+             window=wl.win_len, layers=n_layers, variants="curr+prev", steering="decay",
+             l2="inputs larger than L2 (weights streamed every step)")
+    c.update(extra)
+    return c
 
 
 def _setup(wl, dev, n_layers):
@@ -172,8 +189,9 @@ def run_reference(args, wl, rank, world):
     committed = _oracle_committed(wl, weights, toks, lens, steer)
     times = []
     sample = None
+    budget = 150.0 / (args.warmup + args.steps)      # the whole run ends within a few minutes
     for i in range(args.warmup + args.steps):
-        s = _oracle_sample(wl1, weights, k_log, v_log, toks, lens, steer)
+        s = _oracle_sample(wl1, weights, k_log, v_log, toks, lens, steer, budget_s=budget)
         sample = s["sample"]
         if i >= args.warmup:
             times.append(s["est_step_s"])
@@ -183,7 +201,7 @@ def run_reference(args, wl, rank, world):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=wl.name, batch=wl.batch, layers=n_layers),
+                config=_config(wl, n_layers, committed_per_step=committed),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
@@ -360,11 +378,8 @@ def main():
                 steps=args.steps, warmup=args.warmup, ms_per_step=ms_step, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16" if wl.dtype == "bf16" else "f32",
                 data="synthetic",
-                config=dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
-                            window=wl.win_len, layers=n_layers, variants="curr+prev",
-                            steering="decay", committed_per_step=committed,
-                            l2="inputs larger than L2 (weights streamed every step)",
-                            kernels=args.kernels, status=status_bad),
+                config=_config(wl, n_layers, committed_per_step=committed, kernels=args.kernels,
+                               status=status_bad),
                 clocks=clocks,
                 e2e=dict(value=committed_e2e / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
                          h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
