@@ -97,7 +97,8 @@ struct TcState {
   CUtensorMap map_h, map_lm;
   float* lm_part = nullptr;
   int n_sm = 148, lm_stages = 6;
-  unsigned int* grid_bar = nullptr;  // {count, generation} of the dense chain's grid barrier
+  unsigned int* grid_bar = nullptr;  // arrival counter of the dense chain's grid barrier
+  unsigned int bar_count = 0;        // arrivals the launches of this step have used up so far
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
   bool chain_coop = false;           // launched cooperatively (co-residency guaranteed)
   std::string err;
@@ -347,6 +348,7 @@ bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
 void tc_step_begin(TcState* t) {
   // a step that gave up inside a grid barrier leaves the arrival count behind
   cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), t->s);
+  t->bar_count = 0;
 }
 
 int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_end, const SeqMeta& m,
@@ -378,6 +380,8 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
   p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv;
   p.bar = t->grid_bar; p.status = t->status;
+  p.bar_base = t->bar_count;
+  t->bar_count += (unsigned int)(phase_end - phase_begin - 1) * (unsigned int)t->chain_grid;
 #ifdef DC_CHAIN_TRACE
   static unsigned long long* trace_buf = nullptr;
   static unsigned long long* trace_dev = nullptr;

@@ -68,7 +68,8 @@ struct ChainParams {
   int rows_per_variant;
   __nv_bfloat16 *q, *k, *v;     // q [M, nq*128], k [M, nkv*128], v transposed [nkv*128, ldv]
   int ldv;
-  unsigned int* bar;            // grid barrier words {count, generation}
+  unsigned int* bar;            // grid barrier arrival counter (counts up over a step)
+  unsigned int bar_base;        // its value when this launch starts
   int32_t* status;              // DC_ERR_TIMEOUT lands here; non-zero on entry = do nothing
 #ifdef DC_CHAIN_TRACE
   unsigned long long* trace;    // [cta][16] globaltimer at phase boundaries (tracing build only)
@@ -553,6 +554,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   const int tiles_d = p.d / kChainTile, tiles_f = p.F / kChainTile, tiles_qkv = p.nq + 2 * p.nkv;
   const bool has_qkv = p.phase_end > CH_QKV;
 
+  unsigned int n_barriers = 0;
   for (int ph = p.phase_begin; ph < p.phase_end; ++ph) {
 #ifdef DC_CHAIN_TRACE
     if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph] = ptx::globaltimer();
@@ -600,7 +602,9 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     if (ph + 1 < p.phase_end) {
       __syncthreads();
       if (threadIdx.x == 0) {
-        if (abort_flag == 0 && !ptx::grid_barrier(p.bar, gridDim.x, p.status)) abort_flag = 1;
+        ++n_barriers;
+        if (abort_flag == 0 && !ptx::grid_barrier(p.bar, p.bar_base + n_barriers * gridDim.x, p.status))
+          abort_flag = 1;
         if (abort_flag) atomicExch(p.status, DC_ERR_TIMEOUT);
         ptx::fence_proxy_async_all();
       }

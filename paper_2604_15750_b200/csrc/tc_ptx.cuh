@@ -82,26 +82,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
 }
 
 // ---- grid-wide barrier for persistent kernels whose CTAs are all resident (cooperative launch) --
-// bar[0] counts arrivals, bar[1] is the generation.  The last arriver resets the count and bumps
-// the generation, so the words need no reset between launches.  One thread per CTA calls this
-// after a CTA-wide barrier.  The wait is bounded: returns false after kWaitLimitNs, or as soon as
+// One arrival counter that only counts up: a CTA adds one (fire-and-forget, release) and polls
+// until the counter reaches `target` (acquire).  The host zeroes the word at the start of a step
+// and hands every launch the count its barriers start from.  One thread per CTA calls this after
+// a CTA-wide barrier.  The wait is bounded: returns false after kWaitLimitNs, or as soon as
 // *abort_word (global) is non-zero.
-__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n_ctas,
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int target,
                                              const int* abort_word) {
-  unsigned int gen, old;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(bar + 1) : "memory");
-  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(bar) : "memory");
-  if (old == n_ctas - 1) {
-    asm volatile("st.relaxed.gpu.global.u32 [%0], 0;" ::"l"(bar) : "memory");
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar + 1) : "memory");
-    return true;
-  }
+  asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
   const unsigned long long t0 = globaltimer();
   unsigned int polls = 0;
   while (true) {
-    unsigned int g;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(g) : "l"(bar + 1) : "memory");
-    if (g != gen) return true;
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
     if ((++polls & 0x3f) == 0) {
       int ab;
       asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(ab) : "l"(abort_word) : "memory");
