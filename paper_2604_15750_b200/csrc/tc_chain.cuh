@@ -422,7 +422,7 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
     }
     if (threadIdx.x == 64) { DC_TRACE(2); }
     // the outputs are read through TMA (async proxy) by other CTAs after the grid barrier
-    ptx::fence_proxy_async_all();
+    ptx::fence_proxy_async_global();
     if (threadIdx.x == 64) { DC_TRACE(3); }
   }
 }
@@ -501,7 +501,7 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     __syncthreads();
     if (threadIdx.x == 0) { DC_TRACE(2); }
   }
-  ptx::fence_proxy_async_all();  // `a` is the next phase's TMA operand
+  ptx::fence_proxy_async_global();  // `a` is the next phase's TMA operand
 }
 
 __global__ void __launch_bounds__(kChainThreads, 1)
