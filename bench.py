@@ -41,6 +41,20 @@ def _peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_dense_chain launch (ncu --set full, 4-layer
+# case, see profiles/dense_chain_llada8b_b1.md) and the hash of the kernel sources it belongs to
+_TRAFFIC = dict(workload="llada8b_b1", dram_bytes_per_layer_launch=474.64e6 + 10.30e6,
+                kernel_sha256="9e2a3f821790014d")
+
+
+def _kernel_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("tc_chain.cuh", "tc_ptx.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2604_15750_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
 def _layer_param_count(wl):
     hq, hkv = wl.n_q_heads * wl.head_dim, wl.n_kv_heads * wl.head_dim
     return wl.d_model * (hq + 2 * hkv) + hq * wl.d_model + 3 * wl.d_model * wl.d_ff
@@ -353,15 +367,15 @@ def main():
         ach = flops / (gemm_ms * 1e-3) / 1e12
         roof = dict(bound="tensor", achieved=ach, peak=peaks["bf16_sustained"], unit="TFLOP/s",
                     frac=ach / peaks["bf16_sustained"])
+    # DRAM traffic of the dense chain from the ncu capture summarised in
+    # profiles/dense_chain_llada8b_b1.md (one launch = one layer); valid only for the kernel
+    # sources it was taken with and for this workload, scaled to the launches of one step
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "dense_gemm_traffic.json")
-    if os.path.exists(tpath):
-        try:
-            tj = json.load(open(tpath))
-            traffic = tj["dram_bytes_per_layer"] * n_layers if wl.name == tj.get("workload") else None
-        except Exception:
-            traffic = None
-    roof.update(kernel="dense-layer GEMMs (QKV, O, gate/up, down), all layers of one step",
+    if wl.name == _TRAFFIC["workload"] and _kernel_hash() == _TRAFFIC["kernel_sha256"]:
+        per_layer = _TRAFFIC["dram_bytes_per_layer_launch"]
+        first = per_layer * (wl.d_model * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim) / _layer_param_count(wl)
+        traffic = per_layer * n_layers + first
+    roof.update(kernel="k_dense_chain: dense-layer GEMMs (QKV, O, gate/up, down) + norms, all launches of one step",
                 traffic=traffic, peak_source=peaks["source"] + " (of measured)" if peaks["source"] == "measured"
                 else "fallback (of fallback)", stage_ms={k: round(v, 4) for k, v in stage_ms.items()})
 

@@ -41,41 +41,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-// ---- embedding gather: x[row] = E[token of row] -----------------------------------------------
-// Variant 0 (curr): [last block ; window]; variant 1 (prev): the last block's ids replaced by
-// the mask id, everything else fixed, which makes p_prev = p(Z_k | c) (Section 4.4).
-template <typename T>
-__global__ void k_embed(const T* __restrict__ embed, const int32_t* __restrict__ last_ids,
-                        const int32_t* __restrict__ win_ids, int max_last, int max_window,
-                        int mask_id, int vocab, int d, SeqMeta m, float* __restrict__ x,
-                        int32_t* __restrict__ status) {
-  const int row = blockIdx.x;
-  const int r = row % m.R_cap;
-  const int vb = row / m.R_cap;
-  const int b = vb % m.batch, v = vb / m.batch;
-  const int Lb = m.last_len[b], W = m.win_len[b];
-  int tok = mask_id;
-  if (r < Lb) tok = (v == 0) ? last_ids[b * max_last + r] : mask_id;
-  else if (r < Lb + W) tok = win_ids[b * max_window + (r - Lb)];
-  if (tok < 0 || tok >= vocab) {
-    if (threadIdx.x == 0) status[b] = DC_ERR_INDEX;
-    tok = mask_id;
-  }
-  const T* e = embed + (size_t)tok * d;
-  float* xr = x + (size_t)row * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) xr[i] = to_f<T>(e[i]);
-}
-
-template <typename T>
-void launch_embed(const T* embed, const int32_t* last_ids, const int32_t* win_ids, int max_last,
-                  int max_window, int mask_id, int vocab, int d, const SeqMeta& m, float* x,
-                  int32_t* status, cudaStream_t s) {
-  const int M = m.nv * m.batch * m.R_cap;
-  k_embed<T><<<M, 128, 0, s>>>(embed, last_ids, win_ids, max_last, max_window, mask_id, vocab, d,
-                               m, x, status);
-}
-
-// ---- RMSNorm (with the split-K partial sums of the preceding GEMM folded into x) --------------
+// ---- 4-element vector loads / stores ------------------------------------------------------------
 template <typename T> __device__ __forceinline__ void store4(T* dst, const float (&v)[4]);
 template <> __device__ __forceinline__ void store4<float>(float* dst, const float (&v)[4]) {
   *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
@@ -99,6 +65,46 @@ template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bflo
   v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
 }
 
+// ---- embedding gather: x[row] = E[token of row] -----------------------------------------------
+// Variant 0 (curr): [last block ; window]; variant 1 (prev): the last block's ids replaced by
+// the mask id, everything else fixed, which makes p_prev = p(Z_k | c) (Section 4.4).
+template <typename T>
+__global__ void k_embed(const T* __restrict__ embed, const int32_t* __restrict__ last_ids,
+                        const int32_t* __restrict__ win_ids, int max_last, int max_window,
+                        int mask_id, int vocab, int d, SeqMeta m, float* __restrict__ x,
+                        int32_t* __restrict__ status) {
+  const int row = blockIdx.x;
+  const int r = row % m.R_cap;
+  const int vb = row / m.R_cap;
+  const int b = vb % m.batch, v = vb / m.batch;
+  const int Lb = m.last_len[b], W = m.win_len[b];
+  int tok = mask_id;
+  if (r < Lb) tok = (v == 0) ? last_ids[b * max_last + r] : mask_id;
+  else if (r < Lb + W) tok = win_ids[b * max_window + (r - Lb)];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) status[b] = DC_ERR_INDEX;
+    tok = mask_id;
+  }
+  const T* e = embed + (size_t)tok * d;
+  float* xr = x + (size_t)row * d;
+  // d is a multiple of 4: four elements per thread and step
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float v[4];
+    load4<T>(e + i, v);
+    *reinterpret_cast<float4*>(xr + i) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+template <typename T>
+void launch_embed(const T* embed, const int32_t* last_ids, const int32_t* win_ids, int max_last,
+                  int max_window, int mask_id, int vocab, int d, const SeqMeta& m, float* x,
+                  int32_t* status, cudaStream_t s) {
+  const int M = m.nv * m.batch * m.R_cap;
+  k_embed<T><<<M, 128, 0, s>>>(embed, last_ids, win_ids, max_last, max_window, mask_id, vocab, d,
+                               m, x, status);
+}
+
+// ---- RMSNorm (with the split-K partial sums of the preceding GEMM folded into x) --------------
 // One row per block; d is a multiple of 4.  The row (with the partial sums folded in, in split
 // order, so the result does not depend on the launch shape) is written back to x and normed.
 template <typename T>
@@ -180,7 +186,11 @@ __global__ void k_h_override(const T* __restrict__ h_in, int max_window, int d, 
   if (b >= m.batch || k >= m.win_len[b]) return;  // pad rows were zeroed by the final norm
   const T* src = h_in + (((size_t)b * 2 + v) * max_window + k) * d;
   T* dst = h + (size_t)lrow * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float v4[4];
+    load4<T>(src + i, v4);
+    store4<T>(dst + i, v4);
+  }
 }
 
 template <typename T>

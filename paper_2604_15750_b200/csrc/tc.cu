@@ -253,6 +253,11 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
           2 * n_clusters >= grid && grid >= 2) {
         t->chain_grid = grid;
         t->chain_coop = coop != 0;
+        // DC_CHAIN_COOP=0 launches the same grid without the cooperative attribute (all CTAs are
+        // resident anyway when the GPU runs nothing else; every wait in the kernel is bounded).
+        // Profilers that cannot replay cooperative cluster launches need it.
+        const char* e_ = getenv("DC_CHAIN_COOP");
+        if (e_ && e_[0] == '0') t->chain_coop = false;
       }
     }
     cudaGetLastError();
