@@ -5,7 +5,11 @@ Tolerances (bf16 path: every GEMM input is rounded to bf16, fp32 accumulation on
 in the oracle; fp32 path: no rounding):
   logit-like values (lse, xlogp), confidence, entropy : max relative error 2e-2 (bf16) / 1e-4 (f32)
                                                          with denominator max(|ref|, 1)
-  influence I_k                                         : 1e-3 absolute
+  influence I_k                                         : 1e-3 absolute where the LM-head inputs
+      are the same bits on both sides (fp32 model, or steered LM-head input): then only the fp32
+      accumulation of the KL sum differs.  Through a bf16 stack the logits themselves differ
+      (they are allowed 2e-2 relative), and I_k, a difference of two log-probability sets,
+      inherits that: 1e-3 + 2e-2 * max_k I_k.
 Integer outputs (token ids, block length, selected subset) must be identical unless the deciding
 score lies within the float tolerance of its threshold; those cases are counted and returned.
 """
@@ -166,7 +170,9 @@ def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
             assert e <= rtol, (name, b, e)
         e = np.abs(gpu["influence"][b, :W] - o["influence"]).max()
         worst["influence"] = max(worst["influence"], float(e))
-        assert e <= 1e-3, ("influence", b, e)
+        same_inputs = wl.dtype == "f32" or case.steer is not None
+        itol = 1e-3 if same_inputs else 1e-3 + rtol * float(np.max(o["influence"]))
+        assert e <= itol, ("influence", b, e, itol)
         xg, xo = gpu["xlogp"][b, :W, :W], o["xlogp"]
         cols = np.where(same)[0]
         if len(cols):
