@@ -15,8 +15,10 @@
 // Keys beyond the valid length are masked to -inf in S, and the V^T columns of cached keys
 // beyond ctx_len are zeroed in shared memory (the cache may hold anything there).
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2..5 = softmax / output.
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..9 = softmax / output: two threads per query row (TMEM lane quarter = warp % 4), one
+// for each half of the tile's 128 keys (and of O's 128 columns); they meet once per tile to
+// agree on the row maximum and once at the end to add their row sums.
 #pragma once
 #include "kernels.h"
 #include "tc_ptx.cuh"
@@ -33,11 +35,12 @@ struct AttnParams {
   int32_t* status;
 };
 
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 320;
 constexpr int kHd = 128;
 constexpr int kBK = 128;                       // keys per tile
 constexpr int kSub = 128 * 128;                // bytes of one [128 rows x 64 bf16] sub-tile
 constexpr int kAttnSmem = 2 * kSub /*Q*/ + 2 * 4 * kSub /*2 stages of K and V^T*/ + 2 * 2 * kSub /*2 x P*/ + 1024;
+constexpr int kAttnPrefetch = 4;               // context tiles the L2 prefetch runs ahead of the ring
 constexpr float kRescaleGap = 8.f;             // log2 units the tile maximum may exceed m before m moves
 
 __device__ __forceinline__ float attn_ex2(float x) {
@@ -54,6 +57,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __shared__ uint64_t q_full, kv_full[2], kv_empty[2], s_full[2], s_empty[2], p_full[2], pv_done;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
+  __shared__ float xchg[2][128];   // row maximum / row sum of each key half
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* Qs = smem;
@@ -74,8 +78,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     ptx::mbar_init(&q_full, 1);
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&kv_full[i], 1); ptx::mbar_init(&kv_empty[i], 1);
-      ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], 128);
-      ptx::mbar_init(&p_full[i], 128);
+      ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], 256);
+      ptx::mbar_init(&p_full[i], 256);
     }
     ptx::mbar_init(&pv_done, 1);
     ptx::fence_barrier_init();
@@ -94,8 +98,23 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       ptx::mbar_expect_tx(&q_full, 2 * kSub);
       ptx::tma_load_2d(Qs, &map_q, &q_full, h * kHd, row0 + qt * 128);
       ptx::tma_load_2d(Qs + kSub, &map_q, &q_full, h * kHd + 64, row0 + qt * 128);
+      // With two stages a tile's load can only be issued when the tile two before it has been
+      // consumed, so its full latency sits in the loop; context tiles are therefore prefetched
+      // into L2 kAttnPrefetch tiles ahead (the active tiles were just written: L2-resident).
+      auto prefetch_ctx = [&](int t) {
+        if (t < Tc) {
+          const int j0 = t * kBK;
+          const int krow = (b * p.nkv + g) * p.max_ctx + j0, vrow = (b * p.nkv + g) * kHd;
+          ptx::tma_prefetch_l2_3d(&map_kc, 0, krow, p.layer);
+          ptx::tma_prefetch_l2_3d(&map_kc, 64, krow, p.layer);
+          ptx::tma_prefetch_l2_3d(&map_vc, j0, vrow, p.layer);
+          ptx::tma_prefetch_l2_3d(&map_vc, j0 + 64, vrow, p.layer);
+        }
+      };
+      for (int t = 2; t < 2 + kAttnPrefetch; ++t) prefetch_ctx(t);
       for (int t = 0; t < T; ++t) {
         const int s = t & 1;
+        prefetch_ctx(t + 2 + kAttnPrefetch);
         if (!ptx::mbar_wait(&kv_empty[s], (((uint32_t)t >> 1) & 1u) ^ 1u, &abort_flag)) break;
         uint8_t* Ks = KVs + (size_t)s * 4 * kSub;
         uint8_t* Vs = Ks + 2 * kSub;
@@ -119,39 +138,51 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     if (lane == 0) {
+      // lean issue path: this one thread issues 16 MMAs per key tile, so its own instruction
+      // stream is the critical path; descriptors are built once and advanced by additions
       const uint32_t idesc = ptx::idesc_bf16(128, 128);
-      const uint32_t q_addr = ptx::smem_u32(Qs);
+      const uint64_t hi = ptx::smem_desc_sw128_hi();
+      const uint64_t dq = hi | (uint64_t)(ptx::smem_u32(Qs) >> 4);
+      const uint64_t dk0 = hi | (uint64_t)(ptx::smem_u32(KVs) >> 4);                 // stage 0; stage 1 = + 4*kSub
+      const uint64_t dv0 = dk0 + (2 * kSub >> 4);
+      const uint64_t dp0 = hi | (uint64_t)(ptx::smem_u32(Ps) >> 4);                  // buffer 0; buffer 1 = + 2*kSub
+      const uint32_t b_kv_full = ptx::smem_u32(&kv_full[0]), b_kv_empty = ptx::smem_u32(&kv_empty[0]);
+      const uint32_t b_s_full = ptx::smem_u32(&s_full[0]), b_s_empty = ptx::smem_u32(&s_empty[0]);
+      const uint32_t b_p_full = ptx::smem_u32(&p_full[0]), b_pv_done = ptx::smem_u32(&pv_done);
+      constexpr uint64_t kSubU = kSub >> 4;   // one 64-column sub-tile in descriptor units
       bool ok = ptx::mbar_wait(&q_full, 0, &abort_flag);
       auto issue_qk = [&](int t) {
-        const int s = t & 1;
+        const uint32_t s = (uint32_t)t & 1u;
         const uint32_t ph = ((uint32_t)t >> 1) & 1u;
-        if (!ptx::mbar_wait(&kv_full[s], ph, &abort_flag)) return false;
-        if (!ptx::mbar_wait(&s_empty[s], ph ^ 1u, &abort_flag)) return false;
+        if (!ptx::mbar_wait_a(b_kv_full + 8u * s, ph, &abort_flag)) return false;
+        if (!ptx::mbar_wait_a(b_s_empty + 8u * s, ph ^ 1u, &abort_flag)) return false;
         ptx::tc_fence_after();
-        const uint32_t k_addr = ptx::smem_u32(KVs + (size_t)s * 4 * kSub);
+        const uint64_t dk = dk0 + s * (4 * kSubU);
+        const uint32_t d = tmem_base + s * 128;
+        ptx::umma_bf16(d, dq, dk, idesc, 0u);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kSub + (kk & 3) * 32;
-          ptx::umma_bf16(tmem_base + s * 128, ptx::smem_desc_sw128(q_addr + off),
-                         ptx::smem_desc_sw128(k_addr + off), idesc, kk > 0 ? 1u : 0u);
+        for (int kk = 1; kk < 8; ++kk) {
+          const uint64_t off = (uint64_t)(kk >> 2) * kSubU + (uint64_t)(kk & 3) * 2;
+          ptx::umma_bf16_acc(d, dq + off, dk + off, idesc);
         }
-        ptx::umma_commit(&s_full[s]);
+        ptx::umma_commit_a(b_s_full + 8u * s);
         return true;
       };
       auto issue_pv = [&](int t) {
-        const int s = t & 1;
-        if (!ptx::mbar_wait(&p_full[s], ((uint32_t)t >> 1) & 1u, &abort_flag)) return false;
+        const uint32_t s = (uint32_t)t & 1u;
+        if (!ptx::mbar_wait_a(b_p_full + 8u * s, ((uint32_t)t >> 1) & 1u, &abort_flag)) return false;
         ptx::tc_fence_after();
-        const uint32_t p_addr = ptx::smem_u32(Ps + (size_t)s * 2 * kSub);
-        const uint32_t v_addr = ptx::smem_u32(KVs + (size_t)s * 4 * kSub + 2 * kSub);
+        const uint64_t dp = dp0 + s * (2 * kSubU);
+        const uint64_t dv = dv0 + s * (4 * kSubU);
+        const uint32_t d = tmem_base + 256;
+        ptx::umma_bf16(d, dp, dv, idesc, t > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kSub + (kk & 3) * 32;
-          ptx::umma_bf16(tmem_base + 256, ptx::smem_desc_sw128(p_addr + off),
-                         ptx::smem_desc_sw128(v_addr + off), idesc, (t > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 1; kk < 8; ++kk) {
+          const uint64_t off = (uint64_t)(kk >> 2) * kSubU + (uint64_t)(kk & 3) * 2;
+          ptx::umma_bf16_acc(d, dp + off, dv + off, idesc);
         }
-        ptx::umma_commit(&pv_done);
-        ptx::umma_commit(&kv_empty[s]);
+        ptx::umma_commit_a(b_pv_done);
+        ptx::umma_commit_a(b_kv_empty + 8u * s);
         return true;
       };
       if (ok && T > 0) ok = issue_qk(0);
@@ -162,54 +193,66 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     }
   } else {
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;   // which 64 keys of a tile / which 64 columns of O
     const int r = quarter * 32 + lane;  // query row inside the tile = TMEM lane; also V^T row
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    float m_run = -INFINITY, l_run = 0.f;
+    const int kbase = half * 64;
+    float m_run = -INFINITY, l_run = 0.f;   // l_run: this thread's keys only
     bool ok = true;
-    for (int t = 0; t < T && ok; ++t) {
+    // the two threads of a row meet on the named barrier of their lane quarter (64 threads)
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory"); };
+    // Every iteration executes both pair barriers whatever happened (a wait that gave up makes
+    // `ok` false for the whole warp and the work is skipped), so that a failure cannot leave the
+    // partner warp waiting on a barrier.
+    for (int t = 0; t < T; ++t) {
       const int s = t & 1;
       const uint32_t ph = ((uint32_t)t >> 1) & 1u;
       const bool is_ctx = t < Tc;
       const int valid = is_ctx ? min(kBK, P - t * kBK) : min(kBK, R - (t - Tc) * kBK);
-      ok = ptx::mbar_wait(&s_full[s], ph, &abort_flag);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      // the whole score row into registers, then the TMEM buffer is free for Q K^T of tile t+2
-      float sv[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-        ptx::tmem_ld_32x32(t_lane + s * 128 + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(&s_empty[s]);
+      const int vloc = max(0, min(64, valid - kbase));   // valid keys inside this thread's half
+      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[s], ph, &abort_flag));
+      float sv[64];
       float mx = -INFINITY;
+      if (ok) {
+        ptx::tc_fence_after();
+        // this half of the score row into registers, then the TMEM buffer is free for tile t+2
+        ptx::tmem_ld_32x32(t_lane + s * 128 + kbase, *reinterpret_cast<float(*)[32]>(&sv[0]));
+        ptx::tmem_ld_32x32(t_lane + s * 128 + kbase + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&s_empty[s]);
 #pragma unroll
-      for (int j = 0; j < 128; ++j)
-        if (j < valid) mx = fmaxf(mx, sv[j]);
+        for (int j = 0; j < 64; ++j)
+          if (j < vloc) mx = fmaxf(mx, sv[j]);
+      }
+      xchg[half][r] = mx;
+      pair_sync();
+      mx = fmaxf(mx, xchg[half ^ 1][r]);
+      pair_sync();   // the partner has read before the next tile overwrites
+      if (!ok) continue;
       const float m_tile = mx * p.scale_log2;
       // raise the running maximum only when the tile exceeds it by more than the gap
       const bool raise = m_tile > m_run + kRescaleGap;   // true on the first tile (m_run = -inf)
       const float m_new = raise ? m_tile : m_run;
       const float alpha = raise ? attn_ex2(m_run - m_new) : 1.f;  // 0 on the first tile
       float l_tile = 0.f;
-      uint8_t* pbuf = Ps + (size_t)s * 2 * kSub;
+      // keys [kbase, kbase+64) are sub-tile `half` of the P buffer: 8 chunks of 8 keys per row
+      uint8_t* prow = Ps + (size_t)s * 2 * kSub + half * kSub + r * 128;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t packed[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
           const int k0 = c * 32 + j;
-          const float p0 = (k0 < valid) ? attn_ex2(fmaf(sv[k0], p.scale_log2, -m_new)) : 0.f;
-          const float p1 = (k0 + 1 < valid) ? attn_ex2(fmaf(sv[k0 + 1], p.scale_log2, -m_new)) : 0.f;
+          const float p0 = (k0 < vloc) ? attn_ex2(fmaf(sv[k0], p.scale_log2, -m_new)) : 0.f;
+          const float p1 = (k0 + 1 < vloc) ? attn_ex2(fmaf(sv[k0 + 1], p.scale_log2, -m_new)) : 0.f;
           l_tile += p0 + p1;
           __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
           packed[j >> 1] = *reinterpret_cast<uint32_t*>(&pr);
         }
-        // keys [c*32, c*32+32) = 4 chunks of 8 keys; sub-tile c/2, chunk index (c%2)*4 + q
-        uint8_t* prow = pbuf + (c >> 1) * kSub + r * 128;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
-          const int chunk = ((c & 1) * 4 + q4) ^ (r & 7);
+          const int chunk = (c * 4 + q4) ^ (r & 7);
           *reinterpret_cast<uint4*>(prow + (chunk << 4)) =
               make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
         }
@@ -218,47 +261,51 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       m_run = m_new;
       if (is_ctx && valid < kBK) {
         // cached keys beyond ctx_len: zero the V^T columns so that 0 * garbage cannot make NaN
-        ok = ptx::mbar_wait(&kv_full[s], ph, &abort_flag);
-        uint8_t* vrow_base = KVs + (size_t)s * 4 * kSub + 2 * kSub;
-        for (int cidx = valid; cidx < kBK; ++cidx) {
-          const int cc = cidx & 63;
-          uint8_t* a = vrow_base + (cidx >> 6) * kSub + r * 128 + (((cc >> 3) ^ (r & 7)) << 4) + (cc & 7) * 2;
-          *reinterpret_cast<uint16_t*>(a) = 0;
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&kv_full[s], ph, &abort_flag));
+        if (ok) {
+          uint8_t* vrow = KVs + (size_t)s * 4 * kSub + 2 * kSub + half * kSub + r * 128;
+          for (int cc = vloc; cc < 64; ++cc)
+            *reinterpret_cast<uint16_t*>(vrow + (((cc >> 3) ^ (r & 7)) << 4) + (cc & 7) * 2) = 0;
         }
       }
-      if (t > 0) {
+      if (ok && t > 0) {
         // P V of the previous tile is complete: O may be rescaled, and the P buffer this thread
         // writes next (tile t+1) is no longer read
-        ok = ok && ptx::mbar_wait(&pv_done, (uint32_t)(t - 1) & 1u, &abort_flag);
-        if (!ok) break;
-        if (__any_sync(0xffffffffu, raise)) {
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done, (uint32_t)(t - 1) & 1u, &abort_flag));
+        if (ok && __any_sync(0xffffffffu, raise)) {
           ptx::tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             float ov[32];
-            ptx::tmem_ld_32x32(t_lane + 256 + c * 32, ov);
+            ptx::tmem_ld_32x32(t_lane + 256 + kbase + c * 32, ov);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) ov[j] *= alpha;
-            ptx::tmem_st_32x32(t_lane + 256 + c * 32, ov);
+            ptx::tmem_st_32x32(t_lane + 256 + kbase + c * 32, ov);
           }
           ptx::tmem_st_wait();
           ptx::tc_fence_before();
         }
       }
-      ptx::fence_proxy_async_smem();
-      ptx::mbar_arrive(&p_full[s]);
+      if (ok) {
+        ptx::fence_proxy_async_smem();
+        ptx::mbar_arrive(&p_full[s]);
+      }
     }
-    if (ok && T > 0) ok = ptx::mbar_wait(&pv_done, (uint32_t)(T - 1) & 1u, &abort_flag);
+    if (ok && T > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done, (uint32_t)(T - 1) & 1u, &abort_flag));
+    // row sum = the two halves' sums
+    xchg[half][r] = l_run;
+    pair_sync();
+    const float l_all = l_run + xchg[half ^ 1][r];
     const int rq = qt * 128 + r;
     if (ok && T > 0) {
       ptx::tc_fence_after();
-      const float inv = 1.f / l_run;
-      __nv_bfloat16* dst = p.o + (size_t)(row0 + rq) * p.nq * kHd + (size_t)h * kHd;
+      const float inv = 1.f / l_all;
+      __nv_bfloat16* dst = p.o + (size_t)(row0 + rq) * p.nq * kHd + (size_t)h * kHd + kbase;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         float ov[32];
-        ptx::tmem_ld_32x32(t_lane + 256 + c * 32, ov);
+        ptx::tmem_ld_32x32(t_lane + 256 + kbase + c * 32, ov);
         ptx::tmem_ld_wait();
         if (rq < p.m.R_cap) {
 #pragma unroll
