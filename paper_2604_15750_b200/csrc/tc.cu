@@ -293,7 +293,7 @@ static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
   if (stages > 8) stages = 8;
   if (stages < 2) return tfail(t, DC_ERR_UNSUPPORTED, "activation block too large for the smem ring");
   const size_t smem = (size_t)stages * sb + 1024;
-  dim3 grid(tiles, p.nsplit, (p.M + p.BN - 1) / p.BN);
+  dim3 grid(tiles * ((p.M + p.BN - 1) / p.BN), p.nsplit, 1);
   p.status = t->status;
   k_gemm_tc<EPI><<<grid, kGemmThreads, smem, t->s>>>(w0, w1, w2, ma, p, stages);
   cudaError_t e = cudaGetLastError();
@@ -302,7 +302,8 @@ static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
 }
 
 static int pick_split(int tiles, int KB, int max_split) {
-  // enough CTAs to cover the SMs, at least 8 k-blocks each
+  // enough CTAs to cover the SMs, at least 8 k-blocks each; `tiles` counts every CTA of one
+  // split (weight tiles x activation column blocks)
   int s = 148 / tiles;
   if (s < 1) s = 1;
   if (s > max_split) s = max_split;
@@ -465,7 +466,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_OPROJ, 1);
-  p.N = d; p.K = nq * hd; p.nsplit = pick_split(d / kTileN, p.K / kTileK, t->max_split);
+  p.N = d; p.K = nq * hd; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
   rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.wo, L.wo, L.wo, am->o, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
@@ -482,7 +483,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_DOWN, 1);
-  p.N = d; p.K = F; p.nsplit = pick_split(d / kTileN, p.K / kTileK, t->max_split);
+  p.N = d; p.K = F; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
   rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.w_down, L.w_down, L.w_down, am->act, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;

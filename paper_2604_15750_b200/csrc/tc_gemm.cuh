@@ -67,15 +67,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;   // weight tile
-  const int split = blockIdx.y;  // K split
-  const int cblk = blockIdx.z;   // activation column block
+  // Column blocks of one weight tile sit next to each other in the launch order, so that the
+  // CTAs that share a weight tile run together and all but one read it from L2.
+  const int n_cblk = (p.M + p.BN - 1) / p.BN;
+  const int tile = blockIdx.x / n_cblk;   // weight tile
+  const int cblk = blockIdx.x % n_cblk;   // activation column block
+  const int split = blockIdx.y;           // K split
   const int stage_bytes = gemm_stage_bytes(NW, p.BN);
   const int KB = p.K / kTileK;
   const int kb0 = (int)(((long long)split * KB) / p.nsplit);
   const int kb1 = (int)(((long long)(split + 1) * KB) / p.nsplit);
   const int nkb = kb1 - kb0;
-  const uint32_t tmem_cols = (NW == 2) ? 512u : 256u;
+  const uint32_t tmem_cols = 512u;   // two accumulators of up to 256 columns
 
   // which weight matrix and which row of it this tile starts at
   const CUtensorMap* map_w = &map_w0;
@@ -103,44 +106,58 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   ptx::tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
 
+  // One thread issues every TMA load and one every MMA, so their own instruction streams are on
+  // the critical path: slot indices, addresses and descriptors advance by additions only.
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (ptx::elect_one()) {
+    if (lane == 0) {
+      const uint32_t ring0 = ptx::smem_u32(smem);
+      const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
+      const int arow = cblk * p.BN;
+      uint32_t s = 0, ph = 0, slot = ring0;
       for (int i = 0; i < nkb; ++i) {
-        const int s = i % stages;
-        const uint32_t ph = (uint32_t)(i / stages) & 1u;
-        if (!ptx::mbar_wait(&bar_empty[s], ph ^ 1u, &abort_flag)) break;
-        uint8_t* slot = smem + (size_t)s * stage_bytes;
-        ptx::mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
+        if (!ptx::mbar_wait_a(empty0 + 8u * s, ph ^ 1u, &abort_flag)) break;
+        ptx::mbar_expect_tx_a(full0 + 8u * s, (uint32_t)stage_bytes);
         const int kc = (kb0 + i) * kTileK;
-        ptx::tma_load_2d(slot, map_w, &bar_full[s], kc, wrow);
-        if (NW == 2) ptx::tma_load_2d(slot + kTileN * kTileK * 2, &map_w1, &bar_full[s], kc, wrow);
-        ptx::tma_load_2d(slot + NW * kTileN * kTileK * 2, &map_a, &bar_full[s], kc, cblk * p.BN);
+        ptx::tma_load_2d_a(slot, map_w, full0 + 8u * s, kc, wrow);
+        if (NW == 2) ptx::tma_load_2d_a(slot + kTileN * kTileK * 2, &map_w1, full0 + 8u * s, kc, wrow);
+        ptx::tma_load_2d_a(slot + NW * kTileN * kTileK * 2, &map_a, full0 + 8u * s, kc, arow);
+        if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (ptx::elect_one()) {
+    // Two accumulators (TMEM columns 0.. and 256..) alternate so that consecutive MMAs do not
+    // depend on each other: gate / up have one each, the other epilogues get even k-steps in
+    // the first and odd k-steps in the second and add them.
+    if (lane == 0) {
       const uint32_t idesc = ptx::idesc_bf16(kTileN, p.BN);
-      bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
-        const int s = i % stages;
-        const uint32_t ph = (uint32_t)(i / stages) & 1u;
-        ok = ptx::mbar_wait(&bar_full[s], ph, &abort_flag);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        const uint32_t slot = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t dw0 = ptx::smem_desc_sw128(slot);
-        const uint64_t dw1 = ptx::smem_desc_sw128(slot + kTileN * kTileK * 2);
-        const uint64_t da = ptx::smem_desc_sw128(slot + NW * kTileN * kTileK * 2);
+      const uint32_t ring0 = ptx::smem_u32(smem);
+      const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
+      const uint64_t hi = ptx::smem_desc_sw128_hi();
+      uint32_t s = 0, ph = 0, slot = ring0, acc_first = 0;
+      for (int i = 0; i < nkb; ++i) {
+        if (!ptx::mbar_wait_a(full0 + 8u * s, ph, &abort_flag)) break;
+        const uint64_t dw0 = hi | (uint64_t)(slot >> 4);
+        const uint64_t dw1 = dw0 + (kTileN * kTileK * 2 >> 4);
+        const uint64_t da = dw0 + (NW * kTileN * kTileK * 2 >> 4);
+        if (NW == 2) {
+          ptx::umma_bf16(tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16(tmem_base + 256, dw1, da, idesc, acc_first);
 #pragma unroll
-        for (int kk = 0; kk < kTileK / 16; ++kk) {
-          const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
-          // +32 bytes per 16 bf16 along K = +2 in the 16-byte units of the start address
-          ptx::umma_bf16(tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc, acc);
-          if (NW == 2) ptx::umma_bf16(tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc, acc);
+          for (int kk = 1; kk < kTileK / 16; ++kk) {
+            ptx::umma_bf16_acc(tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
+            ptx::umma_bf16_acc(tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
+          }
+        } else {
+          ptx::umma_bf16(tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16(tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
+          ptx::umma_bf16_acc(tmem_base, dw0 + 4, da + 4, idesc);
+          ptx::umma_bf16_acc(tmem_base + 256, dw0 + 6, da + 6, idesc);
         }
-        ptx::umma_commit(&bar_empty[s]);  // slot free once these MMAs have read it
+        acc_first = 1;
+        ptx::umma_commit_a(empty0 + 8u * s);  // slot free once these MMAs have read it
+        if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
       }
       ptx::umma_commit(&bar_acc);         // accumulators complete
     }
@@ -165,6 +182,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           for (int j = 0; j < 16; ++j) { acc[j] = a16[j]; acc[16 + j] = 0.f; }
         }
         ptx::tmem_ld_wait();
+        if (EPI != GEMM_EPI_SWIGLU) {
+          // odd k-steps went to the second accumulator
+          float odd[32];
+          if (width == 32) ptx::tmem_ld_32x32(t_lane + 256 + c0, odd);
+          else {
+            float a16[16];
+            ptx::tmem_ld_32x16(t_lane + 256 + c0, a16);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { odd[j] = a16[j]; odd[16 + j] = 0.f; }
+          }
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] += odd[j];
+        }
         if (EPI == GEMM_EPI_PARTIAL) {
           float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kTileN + f);
 #pragma unroll
