@@ -501,11 +501,13 @@ int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id,
   p.m = m; p.V = g.vocab; p.K = g.d_model; p.mask_id = forbid ? mask_id : -1;
   p.part = t->lm_part; p.status = t->status;
   const int ntiles = (g.vocab + 127) / 128;
-  const int nctas = ntiles < t->n_sm ? ntiles : t->n_sm;
   const int groups = m.npos_pad / m.G;
-  dim3 grid(nctas, groups);
-  k_lmhead_tc<<<grid, kLmThreads, t->lm_stages * kLmStageBytes + 1024, t->s>>>(t->map_h, t->map_lm,
-                                                                               p, t->lm_stages);
+  int nctas = t->n_sm / groups;             // vocabulary slices: one resident CTA per (group, slice)
+  if (nctas < 1) nctas = 1;
+  if (nctas > ntiles) nctas = ntiles;
+  p.ngroups = groups;
+  k_lmhead_tc<<<groups * nctas, kLmThreads, t->lm_stages * kLmStageBytes + 1024, t->s>>>(t->map_h, t->map_lm,
+                                                                                      p, t->lm_stages);
   const int npos = m.batch * m.W_cap;
   k_lm_combine<<<(npos + 3) / 4, 128, 0, t->s>>>(t->lm_part, nctas, m, ws_pred, ws_conf, ws_ent,
                                                  ws_infl, ws_lse, out);
@@ -656,9 +658,12 @@ extern "C" int dc_signals_static(const dc_signals_in* in, const dc_signals_out* 
   p.m = m; p.V = in->vocab; p.K = in->d_model; p.mask_id = in->forbid_mask_pred ? in->mask_id : -1;
   p.part = part; p.status = word;
   const int ntiles = (in->vocab + 127) / 128;
-  const int nctas = ntiles < sd.n_sm ? ntiles : sd.n_sm;
-  dim3 grid(nctas, m.npos_pad / m.G);
-  k_lmhead_tc<<<grid, kLmThreads, sd.lm_stages * kLmStageBytes + 1024, s>>>(map_h, map_lm, p, sd.lm_stages);
+  const int groups = m.npos_pad / m.G;
+  int nctas = sd.n_sm / groups;
+  if (nctas < 1) nctas = 1;
+  if (nctas > ntiles) nctas = ntiles;
+  p.ngroups = groups;
+  k_lmhead_tc<<<groups * nctas, kLmThreads, sd.lm_stages * kLmStageBytes + 1024, s>>>(map_h, map_lm, p, sd.lm_stages);
   SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, in->max_window};
   k_lm_combine<<<(npos + 3) / 4, 128, 0, s>>>(part, nctas, m, ws_pred, ws_conf, ws_ent, ws_infl, ws_lse, so);
   k_static_status<<<1, 32, 0, s>>>(word, out->status, in->batch);

@@ -11,9 +11,12 @@
 // Orientation: the 128 TMEM lanes are LM rows of one group ([G curr rows ; G prev rows]), the
 // TMEM columns are 128 vocabulary entries, so each thread scans its own row serially; the only
 // exchange is z' from the prev row's thread to the curr row's thread, through shared memory.
-// CTAs are persistent over vocabulary tiles (tile = blockIdx.x, += gridDim.x) with two TMEM
-// accumulators, so the statistics of tile j overlap the MMAs of tile j+1.  Each CTA writes one
-// partial record per row; k_lm_combine merges the records of all CTAs.
+// CTAs are persistent over vocabulary tiles (tile = blockIdx.x, += gridDim.x), two tiles at a
+// time: the MMAs of a pair alternate between two TMEM accumulators (a chain of MMAs into one
+// accumulator issues at 151 clk per MMA, two alternating ones at 86 clk for N = 128, and both
+// MMAs of a k-step share the h operand), and two such pairs of accumulators exist, so that the
+// statistics of one pair overlap the MMAs of the next.  Each CTA writes one partial record per
+// row; k_lm_combine merges the records of all CTAs.
 #pragma once
 #include "kernels.h"
 #include "tc_ptx.cuh"
@@ -24,12 +27,13 @@ struct LmParams {
   SeqMeta m;
   int V, K;          // vocabulary size, d_model
   int mask_id;       // skipped when >= 0
-  float* part;       // [groups][gridDim.x][128][8]
+  int ngroups;       // groups of LM rows; gridDim.x = ngroups * vocabulary slices
+  float* part;       // [groups][slices][128][8]
   int32_t* status;
 };
 
 constexpr int kLmThreads = 192;
-constexpr int kLmStageBytes = 2 * 128 * 64 * 2;  // h tile + W tile
+constexpr int kLmStageBytes = 3 * 128 * 64 * 2;  // h tile + W tiles of the two vocabulary tiles of a pair
 constexpr float kLog2e = 1.4426950408889634f;
 
 __global__ void __launch_bounds__(kLmThreads, 1)
@@ -43,10 +47,15 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int grp = blockIdx.y;
+  // CTA -> (group of LM rows, vocabulary slice), groups fastest: the CTAs that stream the same
+  // vocabulary tiles for different groups run at the same time, so a tile crosses HBM once and is
+  // served to the other groups from L2
+  const int grp = (int)blockIdx.x % p.ngroups;
+  const int slice = (int)blockIdx.x / p.ngroups, nslices = (int)gridDim.x / p.ngroups;
   const int KB = p.K / 64;
   const int ntiles = (p.V + 127) / 128;
-  const int my_tiles = (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int my_tiles = (ntiles - slice + nslices - 1) / nslices;
+  const int my_pairs = (my_tiles + 1) / 2;
   const int G = p.m.G, nv = p.m.nv;
 
   if (threadIdx.x == 0) {
@@ -58,7 +67,7 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
     ptx::prefetch_tmap(&map_w);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&tmem_base_s, 256);
+    ptx::tmem_alloc(&tmem_base_s, 512);
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before();
@@ -66,48 +75,69 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
   ptx::tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
 
+  // (lean single-thread loops: addresses and descriptors advance by additions only)
   if (warp == 0) {
-    if (ptx::elect_one()) {
-      int it = 0;
+    if (lane == 0) {
+      const uint32_t ring0 = ptx::smem_u32(smem);
+      const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
+      const uint64_t pol_w = ptx::l2_policy_evict_first();
+      uint32_t s = 0, ph = 0, slot = ring0;
       bool ok = true;
-      for (int j = 0; j < my_tiles && ok; ++j) {
-        const int vrow = ((int)blockIdx.x + j * (int)gridDim.x) * 128;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (uint32_t)(it / stages) & 1u;
-          ok = ptx::mbar_wait(&bar_empty[s], ph ^ 1u, &abort_flag);
+      for (int q = 0; q < my_pairs && ok; ++q) {
+        // second tile of the pair may lie beyond the vocabulary: the load is zero-filled there
+        // and the epilogue skips ids >= V
+        const int vrow0 = (slice + (2 * q) * nslices) * 128;
+        const int vrow1 = (slice + (2 * q + 1) * nslices) * 128;
+        const bool two = 2 * q + 1 < my_tiles;
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = ptx::mbar_wait_a(empty0 + 8u * s, ph ^ 1u, &abort_flag);
           if (!ok) break;
-          uint8_t* slot = smem + (size_t)s * kLmStageBytes;
-          ptx::mbar_expect_tx(&bar_full[s], kLmStageBytes);
-          ptx::tma_load_2d(slot, &map_h, &bar_full[s], kb * 64, grp * nv * G);
-          ptx::tma_load_2d(slot + 128 * 64 * 2, &map_w, &bar_full[s], kb * 64, vrow);
+          const uint32_t bar = full0 + 8u * s;
+          ptx::mbar_expect_tx_a(bar, two ? (uint32_t)kLmStageBytes : (uint32_t)(2 * 128 * 64 * 2));
+          ptx::tma_load_2d_a(slot, &map_h, bar, kb * 64, grp * nv * G);
+          ptx::tma_load_2d_hint_a(slot + 128 * 64 * 2, &map_w, bar, kb * 64, vrow0, pol_w);
+          if (two) ptx::tma_load_2d_hint_a(slot + 2 * 128 * 64 * 2, &map_w, bar, kb * 64, vrow1, pol_w);
+          if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)kLmStageBytes;
         }
       }
     }
   } else if (warp == 1) {
-    if (ptx::elect_one()) {
+    if (lane == 0) {
       const uint32_t idesc = ptx::idesc_bf16(128, 128);
-      int it = 0;
+      const uint32_t ring0 = ptx::smem_u32(smem);
+      const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
+      const uint64_t hi = ptx::smem_desc_sw128_hi();
+      uint32_t s = 0, ph = 0, slot = ring0;
       bool ok = true;
-      for (int j = 0; j < my_tiles && ok; ++j) {
-        const int buf = j & 1;
-        ok = ptx::mbar_wait(&acc_empty[buf], (((uint32_t)j >> 1) & 1u) ^ 1u, &abort_flag);
+      for (int q = 0; q < my_pairs && ok; ++q) {
+        const int buf = q & 1;
+        const bool two = 2 * q + 1 < my_tiles;
+        ok = ptx::mbar_wait(&acc_empty[buf], (((uint32_t)q >> 1) & 1u) ^ 1u, &abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (uint32_t)(it / stages) & 1u;
-          ok = ptx::mbar_wait(&bar_full[s], ph, &abort_flag);
+        const uint32_t d0 = tmem_base + buf * 256, d1 = d0 + 128;
+        uint32_t acc_first = 0;
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = ptx::mbar_wait_a(full0 + 8u * s, ph, &abort_flag);
           if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t slot = ptx::smem_u32(smem + (size_t)s * kLmStageBytes);
-          const uint64_t dh = ptx::smem_desc_sw128(slot);
-          const uint64_t dw = ptx::smem_desc_sw128(slot + 128 * 64 * 2);
+          const uint64_t dh = hi | (uint64_t)(slot >> 4);
+          const uint64_t dw0 = dh + (128 * 64 * 2 >> 4), dw1 = dh + (2 * 128 * 64 * 2 >> 4);
+          if (two) {
+            ptx::umma_bf16(d0, dh, dw0, idesc, acc_first);
+            ptx::umma_bf16(d1, dh, dw1, idesc, acc_first);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            ptx::umma_bf16(tmem_base + buf * 128, dh + 2 * kk, dw + 2 * kk, idesc,
-                           (kb > 0 || kk > 0) ? 1u : 0u);
-          ptx::umma_commit(&bar_empty[s]);
+            for (int kk = 1; kk < 4; ++kk) {
+              ptx::umma_bf16_acc(d0, dh + 2 * kk, dw0 + 2 * kk, idesc);
+              ptx::umma_bf16_acc(d1, dh + 2 * kk, dw1 + 2 * kk, idesc);
+            }
+          } else {
+            ptx::umma_bf16(d0, dh, dw0, idesc, acc_first);
+#pragma unroll
+            for (int kk = 1; kk < 4; ++kk) ptx::umma_bf16_acc(d0, dh + 2 * kk, dw0 + 2 * kk, idesc);
+          }
+          acc_first = 1;
+          ptx::umma_commit_a(empty0 + 8u * s);
+          if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)kLmStageBytes;
         }
         if (ok) ptx::umma_commit(&acc_full[buf]);
       }
@@ -122,16 +152,18 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
     float mt = -INFINITY, S = 0.f, A = 0.f, D = 0.f;
     int idx = 0x7fffffff;
     bool ok = true;
-    for (int j = 0; j < my_tiles && ok; ++j) {
-      const int buf = j & 1;
-      const int v0 = ((int)blockIdx.x + j * (int)gridDim.x) * 128;
-      ok = ptx::mbar_wait(&acc_full[buf], ((uint32_t)j >> 1) & 1u, &abort_flag);
+    for (int q = 0; q < my_pairs && ok; ++q) {
+      const int buf = q & 1;
+      ok = ptx::mbar_wait(&acc_full[buf], ((uint32_t)q >> 1) & 1u, &abort_flag);
       if (!ok) break;
       ptx::tc_fence_after();
+      const int n_in_pair = (2 * q + 1 < my_tiles) ? 2 : 1;
+      for (int w = 0; w < n_in_pair; ++w) {
+      const int v0 = (slice + (2 * q + w) * nslices) * 128;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float z[32];
-        ptx::tmem_ld_32x32(t_lane + buf * 128 + c * 32, z);
+        ptx::tmem_ld_32x32(t_lane + buf * 256 + w * 128 + c * 32, z);
         ptx::tmem_ld_wait();
         float* xb = xch[c & 1];
         if (is_prev) {
@@ -174,17 +206,18 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
           }
         }
       }
+      }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&acc_empty[buf]);
     }
-    float* rec = p.part + (((size_t)grp * gridDim.x + blockIdx.x) * 128 + row) * 8;
+    float* rec = p.part + (((size_t)grp * nslices + slice) * 128 + row) * 8;
     rec[0] = mt; rec[1] = __int_as_float(idx); rec[2] = S; rec[3] = A; rec[4] = D;
   }
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 256);
+    ptx::tmem_dealloc(tmem_base, 512);
   }
   if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, DC_ERR_TIMEOUT);
 }
