@@ -70,7 +70,12 @@ enum { DC_MAX_BATCH = 32, DC_MAX_WINDOW = 256 };
 /* dc_step_in.flags */
 enum {
   DC_STEP_INFLUENCE = 1, /* also run the prev variant and reduce I_k (Eq. 3)                */
-  DC_STEP_BOUNDARY = 2   /* run the boundary rule (Section 4.2) and write block_len         */
+  DC_STEP_BOUNDARY = 2,  /* run the boundary rule (Section 4.2) and write block_len         */
+  DC_STEP_EXPORT_KV = 4  /* append the last decoded block's K / V (curr variant, every layer) to
+                            the caches at keys ctx_len[b] .. ctx_len[b] + last_len[b] - 1: the
+                            library WRITES k_cache / v_cache there (block-wise cache reuse,
+                            Section 4.1 "compatible with existing block-wise cache techniques");
+                            needs ctx_len[b] + last_len[b] <= max_ctx                        */
 };
 
 typedef struct dc_config {
@@ -216,6 +221,53 @@ DC_API int dc_boundary(dc_ctx* ctx, const dc_boundary_in* in, const dc_boundary_
  * high-confidence phase, greedy completion, single-token fallback.  Reads the buffers a
  * previous dc_step wrote (or any caller-made ones). */
 DC_API int dc_select(dc_ctx* ctx, const dc_select_in* in, const dc_select_out* out);
+
+/* ---- the decoding loop around the step (Section 3, Eq. 1-2; Section 4.2 "starting from the
+ * current frontier ...") ---------------------------------------------------------------------- */
+
+/* Eq. (2): y_i <- yhat_i for the selected, still masked positions of the current block
+ * window[0, block_len); remaining[b] = masked positions left in that block. */
+typedef struct dc_commit_in {
+  int32_t batch;
+  int32_t* win_ids;          /* device [batch][max_window], updated in place                  */
+  const int32_t* pred_id;    /* device [batch][max_window]                                    */
+  const uint8_t* sel_mask;   /* device [batch][max_window]                                    */
+  const int32_t* block_len;  /* device [batch]                                                */
+  const int32_t* win_len;    /* host [batch]                                                  */
+} dc_commit_in;
+typedef struct dc_commit_out {
+  int32_t* remaining;        /* device [batch], may be null                                   */
+} dc_commit_out;
+DC_API int dc_commit(dc_ctx* ctx, const dc_commit_in* in, const dc_commit_out* out);
+
+/* Block-wise generation of gen_len tokens per sequence after a cached context, with DepCap's two
+ * decisions at every stage.  Per sequence, repeated until gen_len tokens are decoded:
+ *   boundary step   dc_step over [last decoded block ; L_window masked positions] with the prev
+ *                   variant: I_k, H_k -> next block length L (first block: L = L_min); the last
+ *                   block's K / V are appended to the cache (DC_STEP_EXPORT_KV); the step's own
+ *                   predictions already serve the block: dc_select + dc_commit on [0, L)
+ *   denoising steps dc_step over the block's L positions (no prev variant), dc_select,
+ *                   dc_commit, until the block holds no [MASK]
+ * The host reads block lengths and remaining-mask counts after every step (one small copy and a
+ * stream synchronisation per step).  Sequences advance independently; finished ones idle.
+ * k_cache / v_cache: as in dc_step, holding ctx_len[b] keys of context on entry, with room for
+ * ctx_len[b] + gen_len keys (DC_ERR_SHAPE otherwise); they are extended in place.
+ * max_steps bounds the number of dc_step calls (DC_ERR_TIMEOUT when exceeded; <= 0: 4 * gen_len).
+ * Prefill of the context is not part of this call. */
+typedef struct dc_generate_in {
+  int32_t batch;
+  void* k_cache;             /* device, written                                               */
+  void* v_cache;             /* device, written                                               */
+  const int32_t* ctx_len;    /* host [batch]                                                  */
+  int32_t gen_len;           /* tokens to decode per sequence, >= 1                           */
+  int32_t max_steps;
+} dc_generate_in;
+typedef struct dc_generate_out {
+  int32_t* tokens;           /* HOST [batch][gen_len]                                         */
+  int32_t* block_lens;       /* HOST [batch][gen_len]: lengths of the blocks in order, then 0 */
+  int32_t* nfe;              /* HOST [1]: dc_step calls made (model forward evaluations)      */
+} dc_generate_out;
+DC_API int dc_generate(dc_ctx* ctx, const dc_generate_in* in, const dc_generate_out* out);
 
 /* Frees the workspace.  The caller must have synchronised the stream.  Null is a no-op. */
 DC_API int dc_destroy(dc_ctx* ctx);

@@ -380,7 +380,8 @@ def cap_select(conf: np.ndarray, masked: np.ndarray, xlogp: np.ndarray, block_le
 # ------------------------------------------------------------------------------------------
 def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
          last_ids: np.ndarray, win_ids: np.ndarray, remain_len: int,
-         influence: bool = True, h_final=None, n_layers: int | None = None) -> dict:
+         influence: bool = True, h_final=None, n_layers: int | None = None,
+         return_kv: bool = False) -> dict:
     """All per-step outputs for one sequence.
 
     curr variant rows = last decoded block followed by the window; prev variant = the same
@@ -394,7 +395,12 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
         k_ctx, v_ctx = k_ctx[:, :, :ctx_len, :], v_ctx[:, :, :ctx_len, :]
     if h_final is None:
         tok_curr = np.concatenate([last_ids, win_ids]).astype(np.int64)
-        x = forward(cfg, w, tok_curr, ctx_len, k_ctx, v_ctx, n_layers=n_layers)
+        x = forward(cfg, w, tok_curr, ctx_len, k_ctx, v_ctx, n_layers=n_layers,
+                    return_kv=return_kv)
+        kv_last = None
+        if return_kv:  # K / V of the last decoded block's rows, as this (curr) forward made them
+            x, kv = x
+            kv_last = [(k[:Lb], v[:Lb]) for k, v in kv]
         h_curr = final_hidden(cfg, w, x[Lb:])
         h_prev = None
         if have_prev:
@@ -403,6 +409,7 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
             xp = forward(cfg, w, tok_prev, ctx_len, k_ctx, v_ctx, n_layers=n_layers)
             h_prev = final_hidden(cfg, w, xp[Lb:])
     else:
+        kv_last = None
         h_curr = _gemm_in(h_final[0], cfg)
         h_prev = _gemm_in(h_final[1], cfg) if have_prev else None
     z = logits_of(h_curr, w.lm_head, cfg)
@@ -414,4 +421,81 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
     sel = cap_select(conf, masked, xl, L, cfg.tau_low, cfg.tau_high, cfg.gamma, cfg.cap_mode)
     return dict(pred=pred, conf=conf, entropy=ent, influence=infl, lse=lse, lse_prev=lse_prev,
                 xlogp=xl, block_len=L, score=score, cum_influence=cum_i, cum_score=cum_s,
-                selected=sel, logits=z, logits_prev=zp, h_curr=h_curr, h_prev=h_prev)
+                selected=sel, logits=z, logits_prev=zp, h_curr=h_curr, h_prev=h_prev,
+                kv_last=kv_last)
+
+
+# ------------------------------------------------------------------------------------------
+# the decoding loop around the step (Section 3, Eq. 1-2; Section 4.2; Algorithm 1 per step)
+# ------------------------------------------------------------------------------------------
+def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, gen_len: int,
+             max_window: int, max_steps: int | None = None) -> dict:
+    """Decode gen_len tokens after a cached context, one sequence.
+
+    Every stage (Section 4.2): from the frontier, one forward over the last decoded block
+    followed by L_window = min(L_max, remaining, max_window) masked positions gives I_k and
+    H_k, hence the next block length L (L_min when nothing has been decoded yet).  The last
+    block's K / V from that forward join the cache (block-wise cache reuse, Section 4.1).  The
+    same forward's predictions already serve the new block: Algorithm 1 picks the subset of
+    [0, L) to commit (Eq. 2).  Then the block's L positions are denoised alone - forward,
+    Algorithm 1, Eq. 2 - until no [MASK] is left; the block becomes the last decoded block.
+    Returns tokens [gen_len], block_lens (list), nfe (forwards of the curr variant = steps) and
+    a per-step trace (kind, pred, conf, selected, block_len, score, ids after the commit).
+    """
+    P0 = int(ctx_len)
+    n_l = cfg.n_layers
+    nkv, hd = cfg.n_kv_heads, cfg.head_dim
+    kc = np.zeros((n_l, nkv, P0 + gen_len, hd))
+    vc = np.zeros((n_l, nkv, P0 + gen_len, hd))
+    if P0 > 0:
+        kc[:, :, :P0] = np.asarray(k_ctx, dtype=np.float64)[:, :, :P0]
+        vc[:, :, :P0] = np.asarray(v_ctx, dtype=np.float64)[:, :, :P0]
+    cache = P0
+    last = np.zeros(0, dtype=np.int64)
+    tokens: list[int] = []
+    block_lens: list[int] = []
+    trace: list[dict] = []
+    nfe = 0
+    limit = 4 * gen_len if not max_steps or max_steps <= 0 else max_steps
+    while len(tokens) < gen_len:
+        remaining = gen_len - len(tokens)
+        # ---- boundary step
+        if nfe >= limit:
+            raise RuntimeError("max_steps reached")
+        W = min(cfg.L_max, max_window, remaining)
+        win = np.full(W, cfg.mask_id, dtype=np.int64)
+        r = step(cfg, w, kc, vc, cache, last, win, remaining, influence=True, return_kv=True)
+        nfe += 1
+        for l in range(n_l):        # the last block moves into the cache
+            k_l, v_l = r["kv_last"][l]
+            for j in range(len(last)):
+                kc[l, :, cache + j] = k_l[j]
+                vc[l, :, cache + j] = v_l[j]
+        cache += len(last)
+        last = np.zeros(0, dtype=np.int64)
+        L = int(r["block_len"])
+        block_lens.append(L)
+        for i in r["selected"]:
+            win[i] = r["pred"][i]
+        trace.append(dict(kind="boundary", pred=r["pred"], conf=r["conf"], selected=r["selected"],
+                          block_len=L, score=r["score"], ids=win[:L].copy(),
+                          influence=r["influence"], entropy=r["entropy"]))
+        blk = win[:L].copy()
+        # ---- denoising steps inside the block
+        while np.any(blk == cfg.mask_id):
+            if nfe >= limit:
+                raise RuntimeError("max_steps reached")
+            r = step(cfg, w, kc, vc, cache, last, blk, remaining, influence=False)
+            nfe += 1
+            # the block length is fixed now: Algorithm 1 runs over the whole block
+            masked = blk == cfg.mask_id
+            sel = cap_select(r["conf"], masked, r["xlogp"], L, cfg.tau_low, cfg.tau_high,
+                             cfg.gamma, cfg.cap_mode)
+            for i in sel:
+                blk[i] = r["pred"][i]
+            trace.append(dict(kind="denoise", pred=r["pred"], conf=r["conf"], selected=sel,
+                              block_len=L, ids=blk.copy()))
+        tokens.extend(int(t) for t in blk)
+        last = blk.astype(np.int64)
+    return dict(tokens=np.asarray(tokens, dtype=np.int64), block_lens=block_lens, nfe=nfe,
+                trace=trace)

@@ -6,6 +6,7 @@ import ctypes as C
 import os
 from dataclasses import dataclass
 
+import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -13,12 +14,12 @@ _LIB_PATH = os.path.join(_HERE, "libdepcap.so")
 
 DC_OK = 0
 DC_F32, DC_BF16 = 0, 1
-DC_STEP_INFLUENCE, DC_STEP_BOUNDARY = 1, 2
+DC_STEP_INFLUENCE, DC_STEP_BOUNDARY, DC_STEP_EXPORT_KV = 1, 2, 4
 DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
                "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
-           "dc_debug_logits", "dc_step_profiled", "dc_signals_static"]
+           "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate"]
 
 
 class DepCapError(RuntimeError):
@@ -85,6 +86,24 @@ class dc_select_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("sel_mask", "sel_idx", "sel_count")]
 
 
+class dc_commit_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("win_ids", C.c_void_p), ("pred_id", C.c_void_p),
+                ("sel_mask", C.c_void_p), ("block_len", C.c_void_p), ("win_len", _I32P)]
+
+
+class dc_commit_out(C.Structure):
+    _fields_ = [("remaining", C.c_void_p)]
+
+
+class dc_generate_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("ctx_len", _I32P), ("gen_len", C.c_int32), ("max_steps", C.c_int32)]
+
+
+class dc_generate_out(C.Structure):
+    _fields_ = [("tokens", _I32P), ("block_lens", _I32P), ("nfe", _I32P)]
+
+
 class dc_signals_in(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("d_model", "vocab", "mask_id", "forbid_mask_pred", "batch",
                                          "max_window")] + \
@@ -120,6 +139,9 @@ def load_library(path: str | None = None):
     lib_.dc_select.argtypes = [C.c_void_p, C.POINTER(dc_select_in), C.POINTER(dc_select_out)]
     lib_.dc_signals_static.argtypes = [C.POINTER(dc_signals_in), C.POINTER(dc_signals_out),
                                        C.c_void_p]
+    lib_.dc_commit.argtypes = [C.c_void_p, C.POINTER(dc_commit_in), C.POINTER(dc_commit_out)]
+    lib_.dc_generate.argtypes = [C.c_void_p, C.POINTER(dc_generate_in),
+                                 C.POINTER(dc_generate_out)]
     lib_.dc_destroy.argtypes = [C.c_void_p]
     lib_.dc_debug_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
     lib_.dc_last_error.argtypes = [C.c_void_p]
@@ -274,13 +296,15 @@ class DepCap:
 
     # -- dc_step ---------------------------------------------------------------------------
     def _step_structs(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len,
-                      remain_len, influence=True, boundary=True, h_final=None, want_xlogp=True):
+                      remain_len, influence=True, boundary=True, h_final=None, want_xlogp=True,
+                      export_kv=False):
         B = len(win_len)
         self._keep = (k_cache, v_cache, last_ids, win_ids, h_final,
                       _host_i32(ctx_len, B), _host_i32(last_len, B), _host_i32(win_len, B),
                       _host_i32(remain_len, B))
         si = dc_step_in(batch=B, flags=(DC_STEP_INFLUENCE if influence else 0) |
-                        (DC_STEP_BOUNDARY if boundary else 0),
+                        (DC_STEP_BOUNDARY if boundary else 0) |
+                        (DC_STEP_EXPORT_KV if export_kv else 0),
                         k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
                         ctx_len=C.cast(self._keep[5], _I32P), last_ids=_ptr(last_ids),
                         last_len=C.cast(self._keep[6], _I32P), win_ids=_ptr(win_ids),
@@ -292,10 +316,12 @@ class DepCap:
         return si, so
 
     def step(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len, remain_len,
-             influence=True, boundary=True, h_final=None):
-        """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled."""
+             influence=True, boundary=True, h_final=None, export_kv=False):
+        """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled.
+        export_kv: also append the last block's K / V to the caches (which are then written)."""
         si, so = self._step_structs(k_cache, v_cache, ctx_len, last_ids, last_len, win_ids,
-                                    win_len, remain_len, influence, boundary, h_final)
+                                    win_len, remain_len, influence, boundary, h_final,
+                                    export_kv=export_kv)
         self._check(self._lib.dc_step(self._ctx, C.byref(si), C.byref(so)))
         return self.out
 
@@ -338,6 +364,38 @@ class DepCap:
         so = dc_select_out(**{k: _ptr(v) for k, v in self.sel.items()})
         self._check(self._lib.dc_select(self._ctx, C.byref(si), C.byref(so)))
         return self.sel
+
+    def commit(self, win_ids, win_len, pred_id=None, sel_mask=None, block_len=None):
+        """Eq. (2) in place on win_ids; returns the device tensor of masked positions left."""
+        B = len(win_len)
+        wl_ = _host_i32(win_len, B)
+        pred_id = self.out["pred_id"] if pred_id is None else pred_id
+        sel_mask = self.sel["sel_mask"] if sel_mask is None else sel_mask
+        block_len = self.out["block_len"] if block_len is None else block_len
+        if not hasattr(self, "_remaining"):
+            self._remaining = torch.zeros(self.max_batch, dtype=torch.int32, device=self.device)
+        ci = dc_commit_in(batch=B, win_ids=_ptr(win_ids), pred_id=_ptr(pred_id),
+                          sel_mask=_ptr(sel_mask), block_len=_ptr(block_len),
+                          win_len=C.cast(wl_, _I32P))
+        co = dc_commit_out(remaining=_ptr(self._remaining))
+        self._check(self._lib.dc_commit(self._ctx, C.byref(ci), C.byref(co)))
+        return self._remaining
+
+    def generate(self, k_cache, v_cache, ctx_len, gen_len, max_steps=0):
+        """Block-wise generation (host arrays out): tokens [B, gen_len], block_lens, nfe."""
+        B = len(ctx_len)
+        cl_ = _host_i32(ctx_len, B)
+        tokens = (C.c_int32 * (B * gen_len))()
+        blocks = (C.c_int32 * (B * gen_len))()
+        nfe = (C.c_int32 * 1)()
+        gi = dc_generate_in(batch=B, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                            ctx_len=C.cast(cl_, _I32P), gen_len=gen_len, max_steps=max_steps)
+        go = dc_generate_out(tokens=C.cast(tokens, _I32P), block_lens=C.cast(blocks, _I32P),
+                             nfe=C.cast(nfe, _I32P))
+        self._check(self._lib.dc_generate(self._ctx, C.byref(gi), C.byref(go)))
+        tok = np.ctypeslib.as_array(tokens).reshape(B, gen_len).copy()
+        bl = np.ctypeslib.as_array(blocks).reshape(B, gen_len).copy()
+        return tok, [[int(x) for x in row if x > 0] for row in bl], int(nfe[0])
 
     def debug_logits(self, variant=0):
         out = torch.zeros((self.max_batch, self.max_window, self.vocab), dtype=torch.float32,

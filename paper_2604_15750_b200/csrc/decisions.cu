@@ -276,4 +276,39 @@ void launch_select(const float* conf, const int32_t* win_ids, const float* xlogp
                                         max_window, sel_mask, sel_idx, sel_count);
 }
 
+// ---- commit (Eq. 2): y_i <- yhat_i for the selected positions; masked positions left in the block --
+__global__ void __launch_bounds__(kThreads) k_commit(int32_t* __restrict__ win_ids,
+                                                    const int32_t* __restrict__ pred_id,
+                                                    const uint8_t* __restrict__ sel_mask,
+                                                    const int32_t* __restrict__ block_len, SeqMeta m,
+                                                    int mask_id, int max_window,
+                                                    int32_t* __restrict__ remaining) {
+  __shared__ int red[kThreads / 32];
+  const int b = blockIdx.x, i = threadIdx.x;
+  const int W = m.win_len[b];
+  const int L = min(max(block_len[b], 0), W);
+  int left = 0;
+  if (i < W) {
+    const size_t o = (size_t)b * max_window + i;
+    int id = win_ids[o];
+    if (i < L && id == mask_id && sel_mask[o]) { id = pred_id[o]; win_ids[o] = id; }
+    left = (i < L && id == mask_id) ? 1 : 0;
+  }
+  for (int o = 16; o > 0; o >>= 1) left += __shfl_xor_sync(0xffffffffu, left, o);
+  if ((i & 31) == 0) red[i >> 5] = left;
+  __syncthreads();
+  if (i == 0 && remaining) {
+    int t = 0;
+    for (int w = 0; w < kThreads / 32; ++w) t += red[w];
+    remaining[b] = t;
+  }
+}
+
+void launch_commit(int32_t* win_ids, const int32_t* pred_id, const uint8_t* sel_mask,
+                   const int32_t* block_len, const SeqMeta& m, int mask_id, int max_window,
+                   int32_t* remaining, cudaStream_t s) {
+  k_commit<<<m.batch, kThreads, 0, s>>>(win_ids, pred_id, sel_mask, block_len, m, mask_id, max_window,
+                                        remaining);
+}
+
 }  // namespace dc

@@ -85,6 +85,11 @@ struct dc_ctx {
   int32_t* ws_pred = nullptr;
   float *ws_conf = nullptr, *ws_ent = nullptr, *ws_infl = nullptr, *ws_lse = nullptr;
   TcState* tc = nullptr;
+  // workspace of dc_generate: window / last-block ids, step and selection outputs, counters
+  int32_t *g_win = nullptr, *g_last = nullptr, *g_pred = nullptr, *g_blk = nullptr, *g_cnt = nullptr,
+          *g_idx = nullptr, *g_rem = nullptr, *g_status = nullptr;
+  float *g_conf = nullptr, *g_xlogp = nullptr;
+  uint8_t* g_mask = nullptr;
   SeqMeta last_meta{};
   bool have_logits = false;
   Profiler prof;
@@ -185,6 +190,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
   int nsplit = 0;
   size_t part_stride = 0;
 
+  const bool export_kv = (in->flags & DC_STEP_EXPORT_KV) != 0;
   const bool chain = c->use_tc && tc_chain_ok(c->tc, m);
   if (c->use_tc) tc_step_begin(c->tc);
   if (chain) {
@@ -197,6 +203,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     pf.end();
     if (rc != DC_OK) return fail(c, rc, "dense chain failed: %s", tc_error(c->tc));
     for (int l = 0; l < L; ++l) {
+      if (export_kv) tc_export_kv(c->tc, l, m, (__nv_bfloat16*)in->k_cache, (__nv_bfloat16*)in->v_cache);
       pf.begin(DC_STAGE_ATTN, 1);
       rc = tc_attention(c->tc, l, m, (const __nv_bfloat16*)in->k_cache,
                         (const __nv_bfloat16*)in->v_cache);
@@ -225,7 +232,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
       int rc = tc_layer(c->tc, l, m, c->x, (const __nv_bfloat16*)a,
                         (const __nv_bfloat16*)in->k_cache, (const __nv_bfloat16*)in->v_cache,
                         c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
-                        &part, &nsplit, &part_stride, pf);
+                        &part, &nsplit, &part_stride, pf, export_kv);
       if (rc != DC_OK) return fail(c, rc, "tensor-core layer %d failed: %s", l, tc_error(c->tc));
       continue;
     }
@@ -237,6 +244,9 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
                         EPI_STORE_F32, s);
     launch_rope_store<T>(c->tmp, c->cos_sin, m, nq, nkv, hd, q, k, v, s);
     pf.end();
+    if (export_kv)
+      launch_export_kv<T>(k, v, 0, m, nkv, hd, g.max_ctx, (T*)in->k_cache + (size_t)l * k_layer,
+                          (T*)in->v_cache + (size_t)l * k_layer, s);
     pf.begin(DC_STAGE_ATTN, 1);
     launch_attn_simt<T>(q, k, v, kc, vc, g.max_ctx, m, nq, nkv, hd, o, s);
     pf.end();
@@ -303,7 +313,7 @@ int validate_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, SeqMe
   if (!in || !out) return fail(c, DC_ERR_INVALID_ARG, "null in/out");
   if (!out->status) return fail(c, DC_ERR_INVALID_ARG, "out->status is required");
   if (!in->win_ids || !in->win_len) return fail(c, DC_ERR_INVALID_ARG, "win_ids/win_len null");
-  if (in->flags & ~(DC_STEP_INFLUENCE | DC_STEP_BOUNDARY))
+  if (in->flags & ~(DC_STEP_INFLUENCE | DC_STEP_BOUNDARY | DC_STEP_EXPORT_KV))
     return fail(c, DC_ERR_INVALID_ARG, "unknown flag bits 0x%x", in->flags);
   int rc = build_meta(c, in->batch, in->flags, in->ctx_len, in->last_len, in->win_len,
                       in->remain_len, m);
@@ -316,6 +326,14 @@ int validate_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, SeqMe
   if (any_ctx && (!in->k_cache || !in->v_cache))
     return fail(c, DC_ERR_INVALID_ARG, "ctx_len > 0 but k_cache/v_cache null");
   if (any_last && !in->last_ids) return fail(c, DC_ERR_INVALID_ARG, "last_len > 0 but last_ids null");
+  if ((in->flags & DC_STEP_EXPORT_KV) && any_last) {
+    if (!in->k_cache || !in->v_cache)
+      return fail(c, DC_ERR_INVALID_ARG, "DC_STEP_EXPORT_KV needs k_cache / v_cache");
+    for (int b = 0; b < m->batch; ++b)
+      if (m->ctx_len[b] + m->last_len[b] > c->cfg.max_ctx)
+        return fail(c, DC_ERR_SHAPE, "ctx_len[%d] + last_len[%d] = %d exceeds max_ctx=%d", b, b,
+                    m->ctx_len[b] + m->last_len[b], c->cfg.max_ctx);
+  }
   return DC_OK;
 }
 
@@ -430,6 +448,20 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
   c->ws_ent = ws_alloc<float>(c, nw, &ok);
   c->ws_infl = ws_alloc<float>(c, nw, &ok);
   c->ws_lse = ws_alloc<float>(c, nw, &ok);
+  {
+    const size_t nww = nw * g.max_window;
+    c->g_win = ws_alloc<int32_t>(c, nw, &ok);
+    c->g_last = ws_alloc<int32_t>(c, (size_t)g.max_batch * (g.max_last > 0 ? g.max_last : 1), &ok);
+    c->g_pred = ws_alloc<int32_t>(c, nw, &ok);
+    c->g_conf = ws_alloc<float>(c, nw, &ok);
+    c->g_xlogp = ws_alloc<float>(c, nww, &ok);
+    c->g_mask = ws_alloc<uint8_t>(c, nw, &ok);
+    c->g_idx = ws_alloc<int32_t>(c, nw, &ok);
+    c->g_blk = ws_alloc<int32_t>(c, g.max_batch, &ok);
+    c->g_cnt = ws_alloc<int32_t>(c, g.max_batch, &ok);
+    c->g_rem = ws_alloc<int32_t>(c, g.max_batch, &ok);
+    c->g_status = ws_alloc<int32_t>(c, g.max_batch, &ok);
+  }
   if (c->use_tc) {
     int rc = tc_create(g, c->stream, c->M_max, c->Mlm_max, c->wq, c->wk, c->wv, c->wo, c->w_gate,
                        c->w_up, c->w_down, c->lm_head, (const __nv_bfloat16*)c->h, &c->tc);
@@ -498,6 +530,136 @@ int dc_select(dc_ctx* c, const dc_select_in* in, const dc_select_out* out) {
   launch_select(in->conf, in->win_ids, in->xlogp, in->block_len, m, hp, c->cfg.mask_id,
                 c->cfg.max_window, out->sel_mask, out->sel_idx, out->sel_count, c->stream);
   DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
+int dc_commit(dc_ctx* c, const dc_commit_in* in, const dc_commit_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !in->win_ids || !in->pred_id || !in->sel_mask || !in->block_len || !in->win_len)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument");
+  SeqMeta m;
+  int rc = build_meta(c, in->batch, 0, nullptr, nullptr, in->win_len, nullptr, &m);
+  if (rc != DC_OK) return rc;
+  launch_commit(in->win_ids, in->pred_id, in->sel_mask, in->block_len, m, c->cfg.mask_id,
+                c->cfg.max_window, out ? out->remaining : nullptr, c->stream);
+  DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
+int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !out || !in->ctx_len || !out->tokens || !out->nfe)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument");
+  const dc_config& g = c->cfg;
+  const int B = in->batch, N = in->gen_len, MW = g.max_window;
+  if (B < 1 || B > g.max_batch) return fail(c, DC_ERR_SHAPE, "batch %d outside [1, max_batch=%d]", B, g.max_batch);
+  if (N < 1) return fail(c, DC_ERR_INVALID_ARG, "gen_len must be positive");
+  const int Lw_cap = g.L_max < MW ? g.L_max : MW;       // window positions a boundary step looks at
+  if (g.max_last < Lw_cap) return fail(c, DC_ERR_SHAPE, "max_last=%d cannot hold a block of %d", g.max_last, Lw_cap);
+  for (int b = 0; b < B; ++b) {
+    if (in->ctx_len[b] < 0 || in->ctx_len[b] + N > g.max_ctx)
+      return fail(c, DC_ERR_SHAPE, "ctx_len[%d] + gen_len = %d exceeds max_ctx=%d", b, in->ctx_len[b] + N, g.max_ctx);
+  }
+  if ((!in->k_cache || !in->v_cache)) return fail(c, DC_ERR_INVALID_ARG, "k_cache / v_cache null");
+  const int max_steps = in->max_steps > 0 ? in->max_steps : 4 * N;
+
+  struct Seq { int cache, done, blk, last_len, nblocks; };   // cache: keys in the cache; done: tokens decoded
+  std::vector<Seq> sq(B);
+  std::vector<int32_t> h_ctx(B), h_lastlen(B), h_winlen(B), h_remain(B), h_blk(B), h_rem(B);
+  std::vector<int32_t> h_win((size_t)B * MW), h_last((size_t)B * (g.max_last > 0 ? g.max_last : 1));
+  for (int b = 0; b < B; ++b) sq[b] = Seq{in->ctx_len[b], 0, 0, 0, 0};
+  if (out->block_lens) memset(out->block_lens, 0, sizeof(int32_t) * (size_t)B * N);
+  cudaStream_t s = c->stream;
+  int nfe = 0;
+  while (true) {
+    bool any_open = false, any_boundary = false;
+    for (int b = 0; b < B; ++b) {
+      any_open |= sq[b].done < N;
+      any_boundary |= sq[b].done < N && sq[b].blk == 0;
+    }
+    if (!any_open) break;
+    if (nfe >= max_steps) { *out->nfe = nfe; return fail(c, DC_ERR_TIMEOUT, "max_steps=%d reached", max_steps); }
+    // ---- inputs of this step
+    for (int b = 0; b < B; ++b) {
+      Seq& q = sq[b];
+      h_ctx[b] = q.cache;
+      h_remain[b] = N - q.done > 0 ? N - q.done : 1;
+      if (q.done >= N) {                       // finished: a dummy window of one masked position
+        h_lastlen[b] = 0; h_winlen[b] = 1; h_win[(size_t)b * MW] = g.mask_id;
+      } else if (q.blk == 0) {                 // boundary step: all of the look-ahead window masked
+        const int W = (N - q.done) < Lw_cap ? (N - q.done) : Lw_cap;
+        h_lastlen[b] = q.last_len; h_winlen[b] = W;
+        for (int i = 0; i < W; ++i) h_win[(size_t)b * MW + i] = g.mask_id;
+      } else {                                 // denoising step inside the block: ids live on the device
+        h_lastlen[b] = 0; h_winlen[b] = q.blk;
+      }
+    }
+    for (int b = 0; b < B; ++b)
+      if (sq[b].done >= N || sq[b].blk == 0)
+        cudaMemcpyAsync(c->g_win + (size_t)b * MW, h_win.data() + (size_t)b * MW, sizeof(int32_t) * h_winlen[b],
+                        cudaMemcpyHostToDevice, s);
+    if (any_boundary)
+      cudaMemcpyAsync(c->g_last, h_last.data(), sizeof(int32_t) * h_last.size(), cudaMemcpyHostToDevice, s);
+    dc_step_in si{};
+    si.batch = B;
+    si.flags = any_boundary ? (DC_STEP_INFLUENCE | DC_STEP_BOUNDARY | DC_STEP_EXPORT_KV) : 0;
+    si.k_cache = in->k_cache; si.v_cache = in->v_cache; si.ctx_len = h_ctx.data();
+    si.last_ids = c->g_last; si.last_len = h_lastlen.data();
+    si.win_ids = c->g_win; si.win_len = h_winlen.data(); si.remain_len = h_remain.data();
+    dc_step_out so{};
+    so.pred_id = c->g_pred; so.conf = c->g_conf; so.xlogp = c->g_xlogp; so.status = c->g_status;
+    so.block_len = any_boundary ? c->g_blk : nullptr;
+    int rc = dc_step(c, &si, &so);
+    if (rc != DC_OK) return rc;
+    ++nfe;
+    // sequences inside a block keep their block length; the boundary rule wrote the others'
+    for (int b = 0; b < B; ++b)
+      if (!(sq[b].done < N && sq[b].blk == 0)) {
+        const int32_t keep = sq[b].done >= N ? 1 : sq[b].blk;
+        // pageable source: the call returns once the value has been staged
+        cudaMemcpyAsync(c->g_blk + b, &keep, sizeof(int32_t), cudaMemcpyHostToDevice, s);
+      }
+    dc_select_in se{};
+    se.batch = B; se.conf = c->g_conf; se.win_ids = c->g_win; se.xlogp = c->g_xlogp;
+    se.block_len = c->g_blk; se.win_len = h_winlen.data();
+    dc_select_out seo{c->g_mask, c->g_idx, c->g_cnt};
+    rc = dc_select(c, &se, &seo);
+    if (rc != DC_OK) return rc;
+    dc_commit_in ci{B, c->g_win, c->g_pred, c->g_mask, c->g_blk, h_winlen.data()};
+    dc_commit_out co{c->g_rem};
+    rc = dc_commit(c, &ci, &co);
+    if (rc != DC_OK) return rc;
+    cudaMemcpyAsync(h_blk.data(), c->g_blk, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(h_rem.data(), c->g_rem, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    std::vector<int32_t> h_status(B);
+    cudaMemcpyAsync(h_status.data(), c->g_status, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return fail(c, DC_ERR_CUDA, "stream sync failed in dc_generate");
+    for (int b = 0; b < B; ++b)
+      if (h_status[b] != DC_OK) return fail(c, h_status[b], "device-side status %d in sequence %d", h_status[b], b);
+    // ---- state update
+    for (int b = 0; b < B; ++b) {
+      Seq& q = sq[b];
+      if (q.done >= N) continue;
+      if (q.blk == 0) {                        // this was the boundary step
+        q.cache += q.last_len;                 // the last block now lives in the cache
+        q.last_len = 0;
+        q.blk = h_blk[b];
+        if (out->block_lens) out->block_lens[(size_t)b * N + q.nblocks] = q.blk;
+        ++q.nblocks;
+      }
+      if (h_rem[b] == 0) {                     // block complete: read its ids back
+        if (cudaMemcpyAsync(out->tokens + (size_t)b * N + q.done, c->g_win + (size_t)b * MW,
+                            sizeof(int32_t) * q.blk, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess)
+          return fail(c, DC_ERR_CUDA, "reading a finished block back failed");
+        memcpy(h_last.data() + (size_t)b * g.max_last, out->tokens + (size_t)b * N + q.done, sizeof(int32_t) * q.blk);
+        q.last_len = q.blk;
+        q.done += q.blk;
+        q.blk = 0;
+      }
+    }
+  }
+  *out->nfe = nfe;
   return DC_OK;
 }
 

@@ -103,6 +103,12 @@ template <typename T>
 void launch_xlogp(const T* h, const T* lm_head, const int32_t* ws_pred, const float* ws_lse,
                   int d, const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s);
 
+// appends the curr variant's K / V of the last-block rows to one layer's context cache
+// (k_cache / v_cache: that layer's slice); v_ld != 0: v is transposed with that row pitch
+template <typename T>
+void launch_export_kv(const T* k, const T* v, int v_ld, const SeqMeta& m, int nkv, int hd,
+                      int max_ctx, T* k_cache, T* v_cache, cudaStream_t s);
+
 // ---- decision kernels --------------------------------------------------------------------------
 // influence/entropy rows have stride `ld`; outputs have stride max_window.
 void launch_boundary(const float* influence, const float* entropy, int ld, const SeqMeta& m,
@@ -113,5 +119,11 @@ void launch_select(const float* conf, const int32_t* win_ids, const float* xlogp
                    const int32_t* block_len, const SeqMeta& m, const Hyper& hp, int mask_id,
                    int max_window, uint8_t* sel_mask, int32_t* sel_idx, int32_t* sel_count,
                    cudaStream_t s);
+
+// Eq. (2): win_ids[i] <- pred_id[i] where selected and still masked, inside [0, block_len);
+// remaining[b] = masked positions left in the block (may be null)
+void launch_commit(int32_t* win_ids, const int32_t* pred_id, const uint8_t* sel_mask,
+                   const int32_t* block_len, const SeqMeta& m, int mask_id, int max_window,
+                   int32_t* remaining, cudaStream_t s);
 
 }  // namespace dc

@@ -552,6 +552,41 @@ void launch_xlogp(const T* h, const T* lm_head, const int32_t* ws_pred, const fl
                                                   xlogp);
 }
 
+// ---- export of the last decoded block's K / V into the context cache -----------------------------
+// The curr variant's rotated K and V of rows [0, last_len[b]) (the last decoded block, all of its
+// tokens clean) are appended to the cache of one layer at keys ctx_len[b] + r.  k: [M, nkv*hd];
+// v: row-major [M, nkv*hd] (v_ld = 0) or transposed [nkv*hd, v_ld].
+template <typename T>
+__global__ void k_export_kv(const T* __restrict__ k, const T* __restrict__ v, int v_ld, SeqMeta m,
+                            int nkv, int hd, int max_ctx, T* __restrict__ k_cache,
+                            T* __restrict__ v_cache) {
+  const int b = blockIdx.y, r = blockIdx.x;
+  if (r >= m.last_len[b]) return;
+  const int row = act_row(m, 0, b, r);
+  const int key = m.ctx_len[b] + r;
+  for (int i = threadIdx.x; i < nkv * hd; i += blockDim.x) {
+    const int g = i / hd, e = i % hd;
+    k_cache[(((size_t)b * nkv + g) * max_ctx + key) * hd + e] = k[(size_t)row * nkv * hd + i];
+    const T vv = v_ld ? v[(size_t)i * v_ld + row] : v[(size_t)row * nkv * hd + i];
+    v_cache[(((size_t)b * nkv + g) * hd + e) * max_ctx + key] = vv;
+  }
+}
+
+template <typename T>
+void launch_export_kv(const T* k, const T* v, int v_ld, const SeqMeta& m, int nkv, int hd,
+                      int max_ctx, T* k_cache, T* v_cache, cudaStream_t s) {
+  int maxl = 0;
+  for (int b = 0; b < m.batch; ++b) maxl = max(maxl, m.last_len[b]);
+  if (maxl == 0) return;
+  dim3 grid(maxl, m.batch);
+  k_export_kv<T><<<grid, 256, 0, s>>>(k, v, v_ld, m, nkv, hd, max_ctx, k_cache, v_cache);
+}
+template void launch_export_kv<float>(const float*, const float*, int, const SeqMeta&, int, int, int,
+                                      float*, float*, cudaStream_t);
+template void launch_export_kv<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, int,
+                                              const SeqMeta&, int, int, int, __nv_bfloat16*,
+                                              __nv_bfloat16*, cudaStream_t);
+
 // explicit instantiations
 #define DC_INST(T)                                                                              \
   template void launch_embed<T>(const T*, const int32_t*, const int32_t*, int, int, int, int,   \

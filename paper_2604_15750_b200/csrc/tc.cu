@@ -336,6 +336,13 @@ int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k
   return DC_OK;
 }
 
+void tc_export_kv(TcState* t, int layer, const SeqMeta& m, __nv_bfloat16* k_cache, __nv_bfloat16* v_cache) {
+  const dc_config& g = t->g;
+  const size_t per_layer = (size_t)g.max_batch * g.n_kv_heads * g.max_ctx * g.head_dim;
+  launch_export_kv<__nv_bfloat16>(t->k, t->v, t->ldv, m, g.n_kv_heads, g.head_dim, g.max_ctx,
+                                  k_cache + (size_t)layer * per_layer, v_cache + (size_t)layer * per_layer, t->s);
+}
+
 bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
   const dc_config& g = t->g;
   const int M = m.nv * m.batch * m.R_cap;
@@ -439,7 +446,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
-             StageHook& hook) {
+             StageHook& hook, bool export_kv) {
   const dc_config& g = t->g;
   const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
   const int M = m.nv * m.batch * m.R_cap;
@@ -460,6 +467,8 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   hook.end();
   if (rc != DC_OK) return rc;
 
+  if (export_kv)
+    tc_export_kv(t, layer, m, const_cast<__nv_bfloat16*>(k_cache), const_cast<__nv_bfloat16*>(v_cache));
   hook.begin(DC_STAGE_ATTN, 1);
   rc = tc_attention(t, layer, m, k_cache, v_cache);
   hook.end();

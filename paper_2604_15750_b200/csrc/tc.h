@@ -41,7 +41,7 @@ const char* tc_error(const TcState* t);
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
-             StageHook& hook);
+             StageHook& hook, bool export_kv = false);
 
 // Attention of one layer alone (reads the rotated q / k / transposed v the QKV epilogue wrote).
 int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,
@@ -59,6 +59,10 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
              float* x, const __nv_bfloat16* a, const float* cos_sin, const __nv_bfloat16* g2,
              const __nv_bfloat16* g1, int fold_norm1, const float** part, int* nsplit,
              size_t* part_stride);
+
+// Appends the curr variant's K / V of the last-block rows of `layer` (as the QKV epilogue left
+// them) to the caller's caches (base pointers of the whole caches).
+void tc_export_kv(TcState* t, int layer, const SeqMeta& m, __nv_bfloat16* k_cache, __nv_bfloat16* v_cache);
 
 // LM head fused with the streaming softmax statistics; fills the workspace signal arrays and
 // the caller's outputs.  Never writes logits.
