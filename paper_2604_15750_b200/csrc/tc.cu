@@ -380,6 +380,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   const LayerMaps& Lq = t->layers[qkv_layer < g.n_layers ? qkv_layer : layer];
   maps.wo = L.wo; maps.wg = L.w_gate; maps.wu = L.w_up; maps.wd = L.w_down;
   maps.wq = Lq.wq; maps.wk = Lq.wk; maps.wv = Lq.wv;
+  maps.wo_n = Lq.wo;
   maps.a = am->a; maps.o = am->o; maps.act = am->act;
   ChainParams p{};
   p.M = M; p.BN = BN; p.d = d; p.F = F; p.nq = nq; p.nkv = nkv;
