@@ -78,6 +78,8 @@ struct ActMaps {
   CUtensorMap a, o, act;
 };
 
+constexpr int kFlagWords = 512;    // per-tile hand-over counters of the balanced QKV phase
+
 struct TcState {
   dc_config g{};
   cudaStream_t s = nullptr;
@@ -97,7 +99,9 @@ struct TcState {
   CUtensorMap map_h, map_lm;
   float* lm_part = nullptr;
   int n_sm = 148, lm_stages = 6;
-  unsigned int* grid_bar = nullptr;  // arrival counter of the dense chain's grid barrier
+  unsigned int* grid_bar = nullptr;  // arrival counter of the dense chain's grid barrier, then kFlagWords tile flags
+  unsigned int qkv_launches = 0;     // chain launches of this step that ran a QKV phase
+  bool balance_qkv = true;
   unsigned int bar_count = 0;        // arrivals the launches of this step have used up so far
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
   bool chain_coop = false;           // launched cooperatively (co-residency guaranteed)
@@ -232,9 +236,9 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
   }
   // the persistent dense chain needs every CTA resident at once (cooperative launch)
   {
-    t->grid_bar = talloc<unsigned int>(t, 2, &ok);
+    t->grid_bar = talloc<unsigned int>(t, 2 + kFlagWords, &ok);
     if (!ok) return tfail(t, DC_ERR_NOMEM, "dense-chain workspace allocation failed");
-    cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), s);
+    cudaMemsetAsync(t->grid_bar, 0, (2 + kFlagWords) * sizeof(unsigned int), s);
     int dev = 0, coop = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
@@ -258,6 +262,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
         // Profilers that cannot replay cooperative cluster launches need it.
         const char* e_ = getenv("DC_CHAIN_COOP");
         if (e_ && e_[0] == '0') t->chain_coop = false;
+        e_ = getenv("DC_BALANCE_QKV");   // DC_BALANCE_QKV=0: every QKV tile by its owner alone
+        if (e_ && e_[0] == '0') t->balance_qkv = false;
       }
     }
     cudaGetLastError();
@@ -360,8 +366,9 @@ bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
 
 void tc_step_begin(TcState* t) {
   // a step that gave up inside a grid barrier leaves the arrival count behind
-  cudaMemsetAsync(t->grid_bar, 0, 2 * sizeof(unsigned int), t->s);
+  cudaMemsetAsync(t->grid_bar, 0, (2 + kFlagWords) * sizeof(unsigned int), t->s);
   t->bar_count = 0;
+  t->qkv_launches = 0;
 }
 
 int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_end, const SeqMeta& m,
@@ -394,6 +401,30 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
   p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv;
   p.bar = t->grid_bar; p.status = t->status;
+  // QKV has nq + 2 nkv tiles; when that is fewer than the grid has CTAs, the CTA pairs left over
+  // take a share of every tile's k-blocks
+  p.bal_h = 0;
+  p.tile_flags = t->grid_bar + 2;
+  if (phase_end > CH_QKV) {
+    const int tp = (nq + 2 * nkv) / 2, n_help = t->chain_grid / 2 - tp, KB = d / kChainTileK;
+    if (t->balance_qkv && n_help > 0 && tp <= 2 * n_help && nq + 2 * nkv <= kFlagWords && KB >= 4 &&
+        (size_t)(nq + 2 * nkv) * BN * kChainTile <= (size_t)t->max_split * t->part_stride) {
+      // An owner waits for its helper's sums before its own epilogue, so a helper should be done
+      // (loop and hand-over) when the owner's loop ends.  Both loops run at the rate an SM takes
+      // data in: a k-block is one weight tile (two for a helper pair that serves two tile pairs)
+      // plus this CTA's half of the activations; handing a tile's sums over costs about as long
+      // as taking in 1.8 times their bytes (measured: 5.4 us for two tiles of 96 KB).
+      const double wb = kChainTile * kChainTileK * 2.0, ab = (BN / 2) * kChainTileK * 2.0;
+      const int nt = tp > n_help ? 2 : 1;
+      const double hand = 1.8 * nt * BN * kChainTile * 4.0;
+      const double hf = (KB * (wb + ab) - hand) / ((nt + 1) * wb + 2.0 * ab);
+      int h = (int)(hf + 0.5);
+      if (h < 1) h = 1;
+      if (h > KB - 1) h = KB - 1;
+      p.bal_h = h;
+    }
+    p.flag_target = (unsigned int)(kChainThreads / 32) * ++t->qkv_launches;
+  }
   p.bar_base = t->bar_count;
   t->bar_count += (unsigned int)(phase_end - phase_begin - 1) * (unsigned int)t->chain_grid;
 #ifdef DC_CHAIN_TRACE

@@ -33,10 +33,12 @@
 // CTA of a pair issues the MMAs; TMA loads of both CTAs report to the even CTA's full barrier,
 // tcgen05.commit releases the ring slot in both CTAs.  No load is multicast.
 //
-// Warp roles (256 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
-// owns the TMEM allocation).  All eight warps run the epilogue: warp w reads the TMEM lanes
-// 32 * (w % 4) .. +31 (the only ones it can reach) and the column half w / 4, so two warps share
-// every lane quarter.  All eight warps run the norm phases.
+// Warp roles (512 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1
+// owns the TMEM allocation).  All sixteen warps run the epilogue: warp w reads the TMEM lanes
+// 32 * (w % 4) .. +31 (the only ones it can reach) and the column part w / 4, so four warps share
+// every lane quarter.  The RoPE epilogue is a chain of dependent shared-memory exchanges and
+// barriers: with four warps per scheduler instead of two it takes 7.2 k instead of 12.2 k clocks.
+// All warps run the norm phases.
 #pragma once
 #include "kernels.h"
 #include "tc.h"
@@ -69,6 +71,13 @@ struct ChainParams {
   int rows_per_variant;
   __nv_bfloat16 *q, *k, *v;     // q [M, nq*128], k [M, nkv*128], v transposed [nkv*128, ldv]
   int ldv;
+  // QKV has fewer tiles than the grid has CTAs: the CTA pairs beyond the tiles take the last
+  // bal_h k-blocks of the tiles off the others' hands (0: off) and hand the sums over in `part`
+  // (BN * 128 floats per tile); tile_flags[tile] counts the warps that have done so (16 per
+  // launch, counting up over a step), flag_target is the count that means "this launch's"
+  int bal_h;
+  unsigned int* tile_flags;
+  unsigned int flag_target;
   unsigned int* bar;            // grid barrier arrival counter (counts up over a step)
   unsigned int bar_base;        // its value when this launch starts
   int32_t* status;              // DC_ERR_TIMEOUT lands here; non-zero on entry = do nothing
@@ -77,9 +86,10 @@ struct ChainParams {
 #endif
 };
 
-constexpr int kChainThreads = 256;
-constexpr int kChainRing = 208 * 1024;          // TMA ring
-constexpr int kChainXch = 2 * 128 * 17 * 4;     // RoPE exchange buffers of the QKV epilogue (one per column half)
+constexpr int kChainThreads = 512;
+constexpr int kChainParts = kChainThreads / 128;  // warps per TMEM lane quarter = column parts of the epilogue
+constexpr int kChainRing = 190 * 1024;          // TMA ring
+constexpr int kChainXch = kChainParts * 128 * 17 * 4;  // RoPE exchange buffers of the QKV epilogue (one per column part)
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
@@ -121,10 +131,12 @@ struct GemmPhase {
   int nsplit;                       // K splits
   int KB;                           // k-blocks of 64
   int N;                            // output features (row pitch of the output)
+  int bal_h;                        // k-blocks of every tile that helper CTA pairs compute (0: none)
   // what the producer prefetches into L2 once its own loads are issued: the first pf_kb
   // k-blocks of its unit in the phase named here (tiles == 0: nothing)
   const CUtensorMap *pf_w0, *pf_w1, *pf_w2;
   int pf_tiles, pf_nsplit, pf_KB, pf_kb, pf_t1, pf_t2;  // pf_t1 / pf_t2: first tile of w1 / w2
+  int pf_bal_h;
 };
 
 // CTA-level unit u -> (weight tile, K split).  CTAs 2p and 2p+1 form a pair and must hold adjacent
@@ -133,6 +145,39 @@ __device__ __forceinline__ void chain_unit(int u, int nsplit, int& tile, int& sp
   const int pp = u >> 1;
   tile = (pp / nsplit) * 2 + (u & 1);
   split = pp % nsplit;
+}
+
+// The work item of this CTA in a GEMM phase (there is at most one: the launch conditions keep
+// tiles * nsplit within the grid): weight tile, K split, k-block range, kind.  Without balancing
+// an item is a unit as above.  With balancing (bal_h > 0; one split, fewer tile pairs than CTA
+// pairs, at most two tile pairs per helper pair) CTA pair t < tiles / 2 owns tile pair t and computes
+// its k-blocks [0, KB - bal_h) (ITEM_MAIN); helper pair hp = pair - tiles / 2 computes the k-blocks
+// [KB - bal_h, KB) of tile pair hp and, if there is one, of tile pair hp + n_help (tile2) in the
+// same pass - one activation tile, two weight tiles, one accumulator each, the shape of gate / up -
+// and hands the sums over (ITEM_HELP).
+enum { ITEM_FULL = 0, ITEM_MAIN = 1, ITEM_HELP = 2 };
+struct ChainItem { int tile, tile2, split, kb0, kb1, kind; };
+__device__ __forceinline__ bool chain_item(int tiles, int nsplit, int KB, int bal_h, ChainItem& w) {
+  w.tile2 = -1;
+  if (bal_h == 0) {
+    if ((int)blockIdx.x >= tiles * nsplit) return false;
+    chain_unit(blockIdx.x, nsplit, w.tile, w.split);
+    w.kb0 = (int)(((long long)w.split * KB) / nsplit);
+    w.kb1 = (int)(((long long)(w.split + 1) * KB) / nsplit);
+    w.kind = ITEM_FULL;
+    return true;
+  }
+  const int pair = blockIdx.x >> 1, r = blockIdx.x & 1, tp = tiles >> 1;
+  w.split = 0;
+  if (pair < tp) {
+    w.tile = 2 * pair + r; w.kb0 = 0; w.kb1 = KB - bal_h; w.kind = ITEM_MAIN;
+    return true;
+  }
+  const int n_help = (gridDim.x >> 1) - tp, hp = pair - tp;
+  if (hp >= tp) return false;
+  w.tile = 2 * hp + r; w.kb0 = KB - bal_h; w.kb1 = KB; w.kind = ITEM_HELP;
+  if (hp + n_help < tp) w.tile2 = 2 * (hp + n_help) + r;
+  return true;
 }
 
 enum { CEPI_PARTIAL = 0, CEPI_SWIGLU = 1, CEPI_QKV = 2 };
@@ -159,8 +204,14 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
     __nv_bfloat16* dst = p.act + (size_t)(tile * kChainTile + f) + (size_t)c0 * N;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
+      // silu(g) = g * sigmoid(g) = g * (0.5 + 0.5 * tanh(g / 2)): one special-function
+      // instruction instead of two (exp and reciprocal); this epilogue is bound by that unit
+      // (16 results per clock and SM).  tanh.approx is good to about 2^-11 absolute, the result
+      // is rounded to bf16
       const float gt = v0[j];
-      dst[(size_t)j * N] = __float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * v1[j]);
+      float th;
+      asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * gt));
+      dst[(size_t)j * N] = __float2bfloat16_rn(gt * fmaf(0.5f, th, 0.5f) * v1[j]);
     }
   } else {  // CEPI_QKV
 #pragma unroll
@@ -182,8 +233,8 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
     } else {
       // rotate-half RoPE: feature i < 64 pairs with i + 64, held by the warp two quarters
       // away; the chunk is exchanged through shared memory
+      float* xch = c.xch + half * (128 * 17);   // `half`: the column part of this warp
 #pragma unroll
-      float* xch = c.xch + half * (128 * 17);
       for (int j = 0; j < 16; ++j) xch[f * 17 + j] = v0[j];
       // the 128 threads of this column half meet on their own named barrier (1 or 2)
       asm volatile("bar.sync %0, 128;" ::"r"(half + 1) : "memory");
@@ -216,13 +267,21 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
 template <int EPI>
 __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, const GemmPhase& g,
                                            const int ph) {
-  constexpr int NW = (EPI == CEPI_SWIGLU) ? 2 : 1;
   const int BN = p.BN;
   const int half_rows = BN >> 1;  // activation rows this CTA stages (the pair MMA reads both halves)
-  const int slot_bytes = NW * kChainTile * kChainTileK * 2 + half_rows * kChainTileK * 2;
+  ChainItem w;
+  const bool has = chain_item(g.tiles, g.nsplit, g.KB, g.bal_h, w);
+  // weight tiles per k-block: gate and up, or the two tiles of a helper pair in a balanced QKV
+  const int nw = (EPI == CEPI_SWIGLU) ? 2 : (EPI == CEPI_QKV && has && w.tile2 >= 0) ? 2 : 1;
+  const int slot_bytes = nw * kChainTile * kChainTileK * 2 + half_rows * kChainTileK * 2;
   int stages = kChainRing / slot_bytes;
   if (stages > 8) stages = 8;
-  const int n_units = g.tiles * g.nsplit;
+  // map and first row of a QKV tile (q tiles, then k, then v)
+  auto qkv_src = [&](int tile, const CUtensorMap*& m, int& row) {
+    m = g.w0; row = tile * kChainTile;
+    if (tile >= p.nq + p.nkv) { m = g.w2; row = (tile - p.nq - p.nkv) * kChainTile; }
+    else if (tile >= p.nq) { m = g.w1; row = (tile - p.nq) * kChainTile; }
+  };
 
   if (c.warp == 0) {
     if (c.lane == 0) {
@@ -234,19 +293,15 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       const int arow = (int)c.rank * half_rows;
       uint32_t ps = 0, pslot = ring0;
       const uint64_t pol_w = ptx::l2_policy_evict_first(), pol_a = ptx::l2_policy_evict_last();
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        int tile, split;
-        chain_unit(u, g.nsplit, tile, split);
-        const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
-        const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
-        const CUtensorMap* mw = g.w0;
-        int wrow = tile * kChainTile;
+      if (has) {
+        const CUtensorMap *mw = g.w0, *mw2 = g.w1;
+        int wrow = w.tile * kChainTile, wrow2 = wrow;
         if (EPI == CEPI_QKV) {
-          if (tile >= p.nq + p.nkv) { mw = g.w2; wrow = (tile - p.nq - p.nkv) * kChainTile; }
-          else if (tile >= p.nq) { mw = g.w1; wrow = (tile - p.nq) * kChainTile; }
+          qkv_src(w.tile, mw, wrow);
+          if (nw == 2) qkv_src(w.tile2, mw2, wrow2);
         }
         // lean loop: slot index, addresses and coordinates advance by additions only
-        for (int kb = kb0; kb < kb1; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           const uint32_t par = (c.fill_bits >> ps) & 1u;
           c.fill_bits ^= 1u << ps;
 #ifdef DC_CHAIN_TRACE
@@ -262,42 +317,42 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           if (c.rank == 0) ptx::mbar_expect_tx_a(full0 + 8u * ps, 2u * (uint32_t)slot_bytes);
           const uint32_t bar = full_remote0 + 8u * ps;
           const int kc = kb * kChainTileK;
-          if (kPrefetchAhead > 0 && kb + kPrefetchAhead < kb1) {
+          if (kPrefetchAhead > 0 && kb + kPrefetchAhead < w.kb1) {
             ptx::tma_prefetch_l2_2d(mw, kc + kPrefetchAhead * kChainTileK, wrow);
-            if (NW == 2) ptx::tma_prefetch_l2_2d(g.w1, kc + kPrefetchAhead * kChainTileK, wrow);
+            if (nw == 2) ptx::tma_prefetch_l2_2d(mw2, kc + kPrefetchAhead * kChainTileK, wrow2);
           }
           // weights pass through L2 once (evict first); the activation tile is re-read by every CTA
           // and the small buffers between phases should stay resident (evict last): -5% step time
           ptx::tma_load_2d_pair_hint(pslot, mw, bar, kc, wrow, pol_w);
-          if (NW == 2) ptx::tma_load_2d_pair_hint(pslot + kChainTile * kChainTileK * 2, g.w1, bar, kc, wrow, pol_w);
-          ptx::tma_load_2d_pair_hint(pslot + NW * kChainTile * kChainTileK * 2, g.amap, bar, kc, arow, pol_a);
+          if (nw == 2) ptx::tma_load_2d_pair_hint(pslot + kChainTile * kChainTileK * 2, mw2, bar, kc, wrow2, pol_w);
+          ptx::tma_load_2d_pair_hint(pslot + nw * kChainTile * kChainTileK * 2, g.amap, bar, kc, arow, pol_a);
           if (++ps == (uint32_t)stages) { ps = 0; pslot = ring0; } else pslot += (uint32_t)slot_bytes;
         }
       }
       DC_TRACE(0);
-      // ---------------- L2 prefetch of this CTA's unit in the next GEMM phase ----------------
-      if (ok && g.pf_tiles > 0) {
-        const int pn = g.pf_tiles * g.pf_nsplit;
-        for (int u = blockIdx.x; u < pn; u += gridDim.x) {
-          int tile, split;
-          chain_unit(u, g.pf_nsplit, tile, split);
-          const int kb0 = (int)(((long long)split * g.pf_KB) / g.pf_nsplit);
-          int kb1 = (int)(((long long)(split + 1) * g.pf_KB) / g.pf_nsplit);
-          if (kb1 > kb0 + g.pf_kb) kb1 = kb0 + g.pf_kb;
-          const CUtensorMap* mw = g.pf_w0;
-          int wrow = tile * kChainTile;
-          bool both = g.pf_w1 != nullptr && g.pf_t1 == 0;  // gate and up: same rows of two maps
-          if (!both && g.pf_w2 != nullptr && tile >= g.pf_t2) { mw = g.pf_w2; wrow = (tile - g.pf_t2) * kChainTile; }
-          else if (!both && g.pf_w1 != nullptr && tile >= g.pf_t1) { mw = g.pf_w1; wrow = (tile - g.pf_t1) * kChainTile; }
-          for (int kb = kb0; kb < kb1; ++kb) {
-            ptx::tma_prefetch_l2_2d(mw, kb * kChainTileK, wrow);
-            if (both) ptx::tma_prefetch_l2_2d(g.pf_w1, kb * kChainTileK, wrow);
-          }
+      // ---------------- L2 prefetch of this CTA's item in the next GEMM phase ----------------
+      ChainItem n;
+      if (ok && g.pf_tiles > 0 && chain_item(g.pf_tiles, g.pf_nsplit, g.pf_KB, g.pf_bal_h, n)) {
+        const int kb1 = n.kb1 > n.kb0 + g.pf_kb ? n.kb0 + g.pf_kb : n.kb1;
+        const bool both = g.pf_w1 != nullptr && g.pf_t1 == 0;  // gate and up: same rows of two maps
+        auto src = [&](int tile, const CUtensorMap*& m, int& row) {
+          m = g.pf_w0; row = tile * kChainTile;
+          if (!both && g.pf_w2 != nullptr && tile >= g.pf_t2) { m = g.pf_w2; row = (tile - g.pf_t2) * kChainTile; }
+          else if (!both && g.pf_w1 != nullptr && tile >= g.pf_t1) { m = g.pf_w1; row = (tile - g.pf_t1) * kChainTile; }
+        };
+        const CUtensorMap *m0, *m1 = nullptr;
+        int r0, r1 = 0;
+        src(n.tile, m0, r0);
+        if (both) { m1 = g.pf_w1; r1 = r0; }
+        else if (n.tile2 >= 0) src(n.tile2, m1, r1);
+        for (int kb = n.kb0; kb < kb1; ++kb) {
+          ptx::tma_prefetch_l2_2d(m0, kb * kChainTileK, r0);
+          if (m1 != nullptr) ptx::tma_prefetch_l2_2d(m1, kb * kChainTileK, r1);
         }
       }
     }
   } else if (c.warp == 1) {
-    if (c.lane == 0 && c.rank == 0) {
+    if (c.lane == 0 && c.rank == 0 && has) {
       // ---------------- MMA issuer (even CTA of the pair, for both) ----------------
       const uint32_t idesc = ptx::idesc_bf16(2 * kChainTile, BN);
       bool ok = true;
@@ -305,127 +360,170 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       const uint32_t mfull0 = ptx::smem_u32(&c.full[0]), mempty0 = ptx::smem_u32(&c.empty[0]);
       const uint64_t desc_hi = ptx::smem_desc_sw128_hi();
       uint32_t ms = 0, mslot = mring0;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        int tile, split;
-        chain_unit(u, g.nsplit, tile, split);
-        const int kb0 = (int)(((long long)split * g.KB) / g.nsplit);
-        const int kb1 = (int)(((long long)(split + 1) * g.KB) / g.nsplit);
-        if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
-          ok = ptx::mbar_wait(c.acc_empty, (c.mma_units - 1) & 1u, c.abort_flag);
-          if (!ok) break;
-        }
-        ptx::tc_fence_after();
-        uint32_t acc_first = 0;   // 0 until the first k-block of the unit has been issued
-#ifdef DC_CHAIN_TRACE
-        const long long tl0 = clock64();
-#endif
-        for (int kb = kb0; kb < kb1; ++kb) {
-          const uint32_t par = (c.use_bits >> ms) & 1u;
-          c.use_bits ^= 1u << ms;
-#ifdef DC_CHAIN_TRACE
-          const long long tw0 = clock64();
-#endif
-          ok = ptx::mbar_wait_a(mfull0 + 8u * ms, par, c.abort_flag);
-#ifdef DC_CHAIN_TRACE
-          p.trace[blockIdx.x * 64 + 40 + ph * 4] += (unsigned long long)(clock64() - tw0);
-#endif
-          if (!ok) break;
-          const uint64_t dw0 = desc_hi | (uint64_t)(mslot >> 4);
-          const uint64_t dw1 = dw0 + (kChainTile * kChainTileK * 2 >> 4);
-          const uint64_t da = dw0 + (NW * kChainTile * kChainTileK * 2 >> 4);
-          if (NW == 2) {
-            ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
-            ptx::umma_bf16_pair(c.tmem_base + 256, dw1, da, idesc, acc_first);
-#pragma unroll
-            for (int kk = 1; kk < kChainTileK / 16; ++kk) {
-              ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
-              ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
-            }
-          } else {
-            ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
-            ptx::umma_bf16_pair(c.tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
-            ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 4, da + 4, idesc);
-            ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw0 + 6, da + 6, idesc);
-          }
-          acc_first = 1;
-          ptx::umma_commit_pair_a(mempty0 + 8u * ms);   // frees the slot in both CTAs
-          if (++ms == (uint32_t)stages) { ms = 0; mslot = mring0; } else mslot += (uint32_t)slot_bytes;
-        }
-#ifdef DC_CHAIN_TRACE
-        p.trace[blockIdx.x * 64 + 42 + ph * 4] += (unsigned long long)(clock64() - tl0);
-#endif
-        if (ok) ptx::umma_commit_pair(c.acc_full);  // both epilogues start
-        ++c.mma_units;
+      if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
+        ok = ptx::mbar_wait(c.acc_empty, (c.mma_units - 1) & 1u, c.abort_flag);
       }
+      ptx::tc_fence_after();
+      uint32_t acc_first = 0;   // 0 until the first k-block of the unit has been issued
+#ifdef DC_CHAIN_TRACE
+      const long long tl0 = clock64();
+#endif
+      for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
+        const uint32_t par = (c.use_bits >> ms) & 1u;
+        c.use_bits ^= 1u << ms;
+#ifdef DC_CHAIN_TRACE
+        const long long tw0 = clock64();
+#endif
+        ok = ptx::mbar_wait_a(mfull0 + 8u * ms, par, c.abort_flag);
+#ifdef DC_CHAIN_TRACE
+        p.trace[blockIdx.x * 64 + 40 + ph * 4] += (unsigned long long)(clock64() - tw0);
+#endif
+        if (!ok) break;
+        const uint64_t dw0 = desc_hi | (uint64_t)(mslot >> 4);
+        const uint64_t dw1 = dw0 + (kChainTile * kChainTileK * 2 >> 4);
+        const uint64_t da = dw0 + ((uint64_t)nw * (kChainTile * kChainTileK * 2 >> 4));
+        if (nw == 2) {
+          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16_pair(c.tmem_base + 256, dw1, da, idesc, acc_first);
+#pragma unroll
+          for (int kk = 1; kk < kChainTileK / 16; ++kk) {
+            ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
+            ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
+          }
+        } else {
+          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16_pair(c.tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
+          ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 4, da + 4, idesc);
+          ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw0 + 6, da + 6, idesc);
+        }
+        acc_first = 1;
+        ptx::umma_commit_pair_a(mempty0 + 8u * ms);   // frees the slot in both CTAs
+        if (++ms == (uint32_t)stages) { ms = 0; mslot = mring0; } else mslot += (uint32_t)slot_bytes;
+      }
+#ifdef DC_CHAIN_TRACE
+      p.trace[blockIdx.x * 64 + 42 + ph * 4] += (unsigned long long)(clock64() - tl0);
+#endif
+      if (ok) ptx::umma_commit_pair(c.acc_full);  // both epilogues start
+      ++c.mma_units;
       DC_TRACE(1);
     }
   }
   __syncwarp();
-  {
-    // ---------------- epilogue: all warps; TMEM lane quarter = warp % 4, column half = warp / 4 ----
+  if (has) {
+    // ---------------- epilogue: all warps; TMEM lane quarter = warp % 4, column part = warp / 4 ----
     const int quarter = c.warp & 3;
-    const int half = c.warp >> 2;
-    const int col_mid = ((BN >> 1) + 15) & ~15;      // columns [0, col_mid) and [col_mid, BN)
-    const int col0 = half ? col_mid : 0, col1 = half ? BN : col_mid;
+    const int half = c.warp >> 2;                    // column part 0 .. kChainParts-1
+    const int part_cols = ((BN / 16 + kChainParts - 1) / kChainParts) * 16;
+    const int col0 = min(half * part_cols, BN), col1 = min(col0 + part_cols, BN);
     const int f = quarter * 32 + c.lane;  // feature inside the tile = TMEM lane
     const uint32_t t_lane = c.tmem_base + ((uint32_t)(quarter * 32) << 16);
-    bool ok = true;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      int tile, split;
-      chain_unit(u, g.nsplit, tile, split);
-      // RoPE factors do not depend on the accumulators: fetch them while the MMAs still run
-      const bool rope = EPI == CEPI_QKV && tile < p.nq + p.nkv;
-      RopeBase rb{1.f, 0.f, 1.f, 0.f}, rb_next{1.f, 0.f, 1.f, 0.f};
-      auto rope_base = [&](int c0, RopeBase& r) {
-        int m0 = c0;  // a chunk of 16 rows never straddles the variants (rows_per_variant % 16 == 0)
-        if (m0 >= p.rows_per_variant) m0 -= p.rows_per_variant;  // prev variant: same table
-        const float* cs = p.cos_sin + (size_t)m0 * 128 + (f & 63);
-        r.c = __ldg(cs); r.s = __ldg(cs + 64);
-      };
-      if (rope) {
-        const float* dl = p.cos_sin + (size_t)p.rows_per_variant * 128 + (f & 63);  // step row
-        rb.cd = __ldg(dl); rb.sd = __ldg(dl + 64);
-        rb_next.cd = rb.cd; rb_next.sd = rb.sd;
-        rope_base(col0, rb);
-      }
-      ok = ptx::mbar_wait(c.acc_full, c.units_done & 1u, c.abort_flag);
-      ++c.units_done;
-      if (!ok) break;
+    const int tile = w.tile, split = w.split, kind = w.kind;
+    const bool rope = EPI == CEPI_QKV && kind != ITEM_HELP && tile < p.nq + p.nkv;
+    RopeBase rb{1.f, 0.f, 1.f, 0.f};
+    auto rope_base = [&](int c0, RopeBase& r) {
+      int m0 = c0;  // a chunk of 16 rows never straddles the variants (rows_per_variant % 16 == 0)
+      if (m0 >= p.rows_per_variant) m0 -= p.rows_per_variant;  // prev variant: same table
+      const float* cs = p.cos_sin + (size_t)m0 * 128 + (f & 63);
+      r.c = __ldg(cs); r.s = __ldg(cs + 64);
+    };
+    if (rope) {
+      const float* dl = p.cos_sin + (size_t)p.rows_per_variant * 128 + (f & 63);  // step row
+      rb.cd = __ldg(dl); rb.sd = __ldg(dl + 64);
+    }
+    bool ok = ptx::mbar_wait(c.acc_full, c.units_done & 1u, c.abort_flag);
+    ++c.units_done;
+    if (ok && EPI == CEPI_QKV && kind == ITEM_MAIN) {
+      // the helper pair's part of this tile has been written (its warps have counted up)
+      bool got = true;
+      if (c.lane == 0) got = ptx::flag_wait(p.tile_flags + tile, p.flag_target, c.abort_flag);
+      ok = __shfl_sync(0xffffffffu, (int)got, 0) != 0;   // also orders the lanes' loads behind the acquire
+    }
+#ifdef DC_CHAIN_TRACE
+    const long long tE0 = clock64();
+    const int eslot = (ph == CH_QKV) ? 13 : 47;   // QKV: 13, 14, 15, 43; gate/up: 47, 51, 55, 59
+    if (threadIdx.x == 64 && (ph == CH_QKV || ph == CH_GATEUP)) p.trace[blockIdx.x * 64 + eslot] = ptx::globaltimer();
+#define DC_ETRACE(c0) if (threadIdx.x == 64 && (ph == CH_QKV || ph == CH_GATEUP)) { const int k_ = ((c0) - col0) / 16; \
+      p.trace[blockIdx.x * 64 + (ph == CH_QKV ? (k_ < 2 ? 14 + k_ : 43) : 51 + 4 * k_)] = (unsigned long long)(clock64() - tE0); }
+#else
+#define DC_ETRACE(c0)
+#endif
+    if (ok) {
       ptx::tc_fence_after();
       // 16 columns (activation rows) per step in a rolled loop (the code runs once per unit, so
-      // it must stay small for the instruction cache), two register buffers: the TMEM loads of
-      // the next step are in flight while this one is converted and stored.  BN equals M here
-      // (M is a multiple of 16), so every column is a real row.
-      float a0[16], a1[16], b0[16], b1[16];
-      ptx::tmem_ld_32x16(t_lane + col0, a0);
-      ptx::tmem_ld_32x16(t_lane + 256 + col0, a1);
+      // it must stay small for the instruction cache).  No register double-buffering: the four
+      // warps of a scheduler cover each other's TMEM and memory latencies.  BN equals M here (M
+      // is a multiple of 16), so every column is a real row.
+      float a0[16], a1[16];
+      if (EPI == CEPI_QKV && kind != ITEM_FULL) {
+        // sums handed from a helper pair to the tile's owner, in the order that makes every
+        // access a 16-byte one and every warp access 512 contiguous bytes:
+        // [tile][chunk of 16 rows][4][128 features][4 rows].  The owner adds them to the first
+        // accumulator's registers; a helper stores the sum of its two accumulators, or, with two
+        // tiles, one accumulator per tile.
+        float4* hand = reinterpret_cast<float4*>(p.part + (size_t)tile * BN * kChainTile) + f;
+        float4* hand2 = reinterpret_cast<float4*>(p.part + (size_t)(w.tile2 >= 0 ? w.tile2 : tile) * BN * kChainTile) + f;
+        const bool dual = w.tile2 >= 0;
 #pragma unroll 1
-      for (int c0 = col0; c0 < col1; c0 += 32) {
-        ptx::tmem_ld_wait();
-        if (c0 + 16 < col1) {
-          ptx::tmem_ld_32x16(t_lane + c0 + 16, b0);
-          ptx::tmem_ld_32x16(t_lane + 256 + c0 + 16, b1);
-          if (rope) rope_base(c0 + 16, rb_next);
-        }
-        chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
-        if (c0 + 16 < col1) {
-          ptx::tmem_ld_wait();
-          if (c0 + 32 < col1) {
-            ptx::tmem_ld_32x16(t_lane + c0 + 32, a0);
-            ptx::tmem_ld_32x16(t_lane + 256 + c0 + 32, a1);
-            if (rope) rope_base(c0 + 32, rb);
+        for (int c0 = col0; c0 < col1; c0 += 16) {
+          ptx::tmem_ld_32x16(t_lane + c0, a0);
+          ptx::tmem_ld_32x16(t_lane + 256 + c0, a1);
+          const size_t cq = (size_t)(c0 >> 4) * 4 * kChainTile;   // float4 index of this chunk
+          if (kind == ITEM_HELP) {
+            ptx::tmem_ld_wait();
+            if (dual) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                __stcg(hand + cq + k * kChainTile, make_float4(a0[4 * k], a0[4 * k + 1], a0[4 * k + 2], a0[4 * k + 3]));
+                __stcg(hand2 + cq + k * kChainTile, make_float4(a1[4 * k], a1[4 * k + 1], a1[4 * k + 2], a1[4 * k + 3]));
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                __stcg(hand + cq + k * kChainTile,
+                       make_float4(a0[4 * k] + a1[4 * k], a0[4 * k + 1] + a1[4 * k + 1],
+                                   a0[4 * k + 2] + a1[4 * k + 2], a0[4 * k + 3] + a1[4 * k + 3]));
+            }
+          } else {
+            float4 ha[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) ha[k] = __ldcg(hand + cq + k * kChainTile);
+            if (rope) rope_base(c0, rb);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              a0[4 * k] += ha[k].x; a0[4 * k + 1] += ha[k].y; a0[4 * k + 2] += ha[k].z; a0[4 * k + 3] += ha[k].w;
+            }
+            chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
           }
-          chain_emit<EPI>(c, p, g.N, tile, split, f, c0 + 16, b0, b1, rb_next, half);
+          DC_ETRACE(c0)
+        }
+        if (kind == ITEM_HELP) {
+          __threadfence();
+          __syncwarp();
+          if (c.lane == 0) {
+            ptx::flag_add(p.tile_flags + tile);
+            if (dual) ptx::flag_add(p.tile_flags + w.tile2);
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c0 = col0; c0 < col1; c0 += 16) {
+          ptx::tmem_ld_32x16(t_lane + c0, a0);
+          ptx::tmem_ld_32x16(t_lane + 256 + c0, a1);
+          if (rope) rope_base(c0, rb);
+          ptx::tmem_ld_wait();
+          chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
+          DC_ETRACE(c0)
         }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(c.acc_empty);
     }
     if (threadIdx.x == 64) { DC_TRACE(2); }
-    // the outputs are read through TMA (async proxy) by other CTAs after the grid barrier
-    ptx::fence_proxy_async_global();
-    if (threadIdx.x == 64) { DC_TRACE(3); }
   }
+  // the outputs are read through TMA (async proxy) by other CTAs after the grid barrier
+  ptx::fence_proxy_async_global();
+  if (threadIdx.x == 64) { DC_TRACE(3); }
 }
 
 // x[row] += sum of the partial sums (in split order); out[row] = bf16(rmsnorm(x[row]) * g).
@@ -435,8 +533,9 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
 __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, int nsplit,
                                            const __nv_bfloat16* __restrict__ g, float* red,
                                            const int ph) {
-  const int grp = c.warp >> 2;                     // 0 or 1
-  const int t = threadIdx.x - grp * 128;           // 0..127 inside the group
+  constexpr int kGrp = kChainThreads / 2;          // threads per row
+  const int grp = threadIdx.x / kGrp;              // 0 or 1
+  const int t = threadIdx.x - grp * kGrp;          // index inside the group
   const int d = p.d;
   const int narr = 1 + nsplit;
   float* stage = reinterpret_cast<float*>(c.ring);  // [grp][narr][d], then the gain vector
@@ -464,7 +563,7 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     float ss = 0.f;
     if (live) {
       float* xr = p.x + (size_t)row * d;
-      for (int i = t * 4; i < d; i += 128 * 4) {
+      for (int i = t * 4; i < d; i += kGrp * 4) {
         float4 v = *reinterpret_cast<const float4*>(sx + i);
         if (nsplit > 0) {
           for (int s = 0; s < nsplit; ++s) {
@@ -481,13 +580,15 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (c.lane == 0) red[c.warp] = ss;
     if (threadIdx.x == 0) { DC_TRACE(1); }
-    // group-wide exchange: named barriers 3 and 4, 128 threads each
-    asm volatile("bar.sync %0, 128;" ::"r"(grp + 3) : "memory");
-    const float tot = red[grp * 4] + red[grp * 4 + 1] + red[grp * 4 + 2] + red[grp * 4 + 3];
+    // group-wide exchange: named barriers 5 and 6 (1..4 belong to the QKV epilogue)
+    asm volatile("bar.sync %0, %1;" ::"r"(grp + 5), "n"(kGrp) : "memory");
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGrp / 32; ++i) tot += red[grp * (kGrp / 32) + i];
     if (live) {
       const float inv = rsqrtf(tot / (float)d + p.eps);
       __nv_bfloat16* outr = p.a + (size_t)row * d;
-      for (int i = t * 4; i < d; i += 128 * 4) {
+      for (int i = t * 4; i < d; i += kGrp * 4) {
         const float4 v = *reinterpret_cast<const float4*>(sx + i);
         const uint2 gw = *reinterpret_cast<const uint2*>(sg + i);
         const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw.x);
@@ -511,7 +612,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
   __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc_full, bar_acc_empty, bar_norm;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
-  __shared__ float red[8];
+  __shared__ float red[kChainThreads / 32];
 
   ChainCtx c;
   c.ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -582,7 +683,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         g.w0 = &maps.wd; g.amap = &maps.act; g.tiles = tiles_d; g.nsplit = p.split_down; g.KB = KBf; g.N = p.d;
         if (has_qkv) {
           g.pf_w0 = &maps.wq; g.pf_w1 = &maps.wk; g.pf_w2 = &maps.wv; g.pf_t1 = p.nq; g.pf_t2 = p.nq + p.nkv;
-          g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = kPfQkv;
+          g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = kPfQkv; g.pf_bal_h = p.bal_h;
         }
         chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
         break;
@@ -591,7 +692,7 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         break;
       default:  // CH_QKV
         g.w0 = &maps.wq; g.w1 = &maps.wk; g.w2 = &maps.wv; g.amap = &maps.a; g.tiles = tiles_qkv;
-        g.nsplit = 1; g.KB = KBd; g.N = 0;
+        g.nsplit = 1; g.KB = KBd; g.N = 0; g.bal_h = p.bal_h;
         // attention runs next; meanwhile the O projection of that layer streams into L2 (gate / up
         // of that layer on top of it was measured slower: +2..4% per step for 8..32 k-blocks)
         g.pf_w0 = &maps.wo_n; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_o; g.pf_KB = KBq; g.pf_kb = 64;

@@ -104,6 +104,26 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
   }
 }
 
+// A counter in global memory that producers count up (after a __threadfence) and a consumer
+// waits for, with the same bound as every other wait.
+__device__ __forceinline__ void flag_add(unsigned int* flag) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(flag) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const unsigned int* flag, unsigned int target,
+                                          volatile int* abort_flag) {
+  const unsigned long long t0 = globaltimer();
+  unsigned int polls = 0;
+  while (true) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= target) return true;
+    if ((++polls & 0x3f) == 0) {
+      if (*abort_flag != 0) return false;
+      if (globaltimer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
 // ---- TMA: tiled 2-D / 3-D loads into shared memory, completion on an mbarrier -----------------
 // The innermost coordinate times the element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar,
