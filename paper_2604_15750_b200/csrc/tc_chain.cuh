@@ -88,8 +88,9 @@ struct ChainParams {
 
 constexpr int kChainThreads = 512;
 constexpr int kChainParts = kChainThreads / 128;  // warps per TMEM lane quarter = column parts of the epilogue
-constexpr int kChainRing = 190 * 1024;          // TMA ring
-constexpr int kChainXch = kChainParts * 128 * 17 * 4;  // RoPE exchange buffers of the QKV epilogue (one per column part)
+constexpr int kChainRing = 184 * 1024;          // TMA ring
+constexpr int kXchRow = 20;                     // floats per thread in a RoPE exchange buffer (16 + padding, 16-byte rows)
+constexpr int kChainXch = kChainParts * 128 * kXchRow * 4;  // RoPE exchange buffers of the QKV epilogue (one per column part)
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
@@ -205,14 +206,15 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       // silu(g) = g * sigmoid(g) = g * (0.5 + 0.5 * tanh(g / 2)): one special-function
-      // instruction instead of two (exp and reciprocal); this epilogue is bound by that unit
-      // (16 results per clock and SM).  tanh.approx is good to about 2^-11 absolute, the result
-      // is rounded to bf16
+      // instruction instead of two (exp and reciprocal; that unit gives 16 results per clock and
+      // SM).  tanh.approx is good to about 2^-11 absolute, the result is rounded to bf16
       const float gt = v0[j];
       float th;
       asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * gt));
-      dst[(size_t)j * N] = __float2bfloat16_rn(gt * fmaf(0.5f, th, 0.5f) * v1[j]);
+      v0[j] = gt * fmaf(0.5f, th, 0.5f) * v1[j];
     }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) dst[(size_t)j * N] = __float2bfloat16_rn(v0[j]);
   } else {  // CEPI_QKV
 #pragma unroll
     for (int j = 0; j < 16; ++j) v0[j] += v1[j];
@@ -233,26 +235,35 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
     } else {
       // rotate-half RoPE: feature i < 64 pairs with i + 64, held by the warp two quarters
       // away; the chunk is exchanged through shared memory
-      float* xch = c.xch + half * (128 * 17);   // `half`: the column part of this warp
+      // each thread's 16 values are one padded row of 20 floats: four 16-byte stores, and the
+      // partner's row comes back with four 16-byte loads (no bank conflicts at this stride)
+      float4* xrow = reinterpret_cast<float4*>(c.xch + half * (128 * kXchRow));   // `half`: the column part of this warp
 #pragma unroll
-      for (int j = 0; j < 16; ++j) xch[f * 17 + j] = v0[j];
-      // the 128 threads of this column half meet on their own named barrier (1 or 2)
+      for (int k = 0; k < 4; ++k)
+        xrow[f * (kXchRow / 4) + k] = make_float4(v0[4 * k], v0[4 * k + 1], v0[4 * k + 2], v0[4 * k + 3]);
+      // the 128 threads of this column part meet on their own named barrier (1 .. 4)
       asm volatile("bar.sync %0, 128;" ::"r"(half + 1) : "memory");
       const bool lo = f < 64;
       const bool is_k = tile >= p.nq;
       const int ld = is_k ? p.nkv * 128 : p.nq * 128;
       __nv_bfloat16* dst = (is_k ? p.k + (size_t)((tile - p.nq) * 128 + f)
                                  : p.q + (size_t)(tile * 128 + f)) + (size_t)c0 * ld;
+      float other[16];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 o4 = xrow[(f ^ 64) * (kXchRow / 4) + k];
+        other[4 * k] = o4.x; other[4 * k + 1] = o4.y; other[4 * k + 2] = o4.z; other[4 * k + 3] = o4.w;
+      }
       float cv = rb.c, sv = rb.s;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float other = xch[(f ^ 64) * 17 + j];
-        const float y = lo ? (v0[j] * cv - other * sv) : (v0[j] * cv + other * sv);
-        dst[(size_t)j * ld] = __float2bfloat16_rn(y);
+        v0[j] = lo ? (v0[j] * cv - other[j] * sv) : (v0[j] * cv + other[j] * sv);
         const float cn = cv * rb.cd - sv * rb.sd;
         sv = sv * rb.cd + cv * rb.sd;
         cv = cn;
       }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) dst[(size_t)j * ld] = __float2bfloat16_rn(v0[j]);
       asm volatile("bar.sync %0, 128;" ::"r"(half + 1) : "memory");
     }
   }
@@ -463,6 +474,16 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         float4* hand = reinterpret_cast<float4*>(p.part + (size_t)tile * BN * kChainTile) + f;
         float4* hand2 = reinterpret_cast<float4*>(p.part + (size_t)(w.tile2 >= 0 ? w.tile2 : tile) * BN * kChainTile) + f;
         const bool dual = w.tile2 >= 0;
+        // the owner's loads (helper sums, RoPE factors) are issued one chunk ahead: the warps of
+        // a column part move in step through the exchange barriers, so nothing else would cover
+        // their latency
+        float4 ha[4], hn[4];
+        RopeBase rn = rb;
+        if (kind == ITEM_MAIN && col0 < col1) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ha[k] = __ldcg(hand + (size_t)(col0 >> 4) * 4 * kChainTile + k * kChainTile);
+          if (rope) rope_base(col0, rb);
+        }
 #pragma unroll 1
         for (int c0 = col0; c0 < col1; c0 += 16) {
           ptx::tmem_ld_32x16(t_lane + c0, a0);
@@ -484,16 +505,20 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
                                    a0[4 * k + 2] + a1[4 * k + 2], a0[4 * k + 3] + a1[4 * k + 3]));
             }
           } else {
-            float4 ha[4];
+            if (c0 + 16 < col1) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) ha[k] = __ldcg(hand + cq + k * kChainTile);
-            if (rope) rope_base(c0, rb);
+              for (int k = 0; k < 4; ++k) hn[k] = __ldcg(hand + cq + (4 + k) * kChainTile);
+              if (rope) rope_base(c0 + 16, rn);
+            }
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               a0[4 * k] += ha[k].x; a0[4 * k + 1] += ha[k].y; a0[4 * k + 2] += ha[k].z; a0[4 * k + 3] += ha[k].w;
             }
             chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) ha[k] = hn[k];
+            rb.c = rn.c; rb.s = rn.s;
           }
           DC_ETRACE(c0)
         }
@@ -506,13 +531,16 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           }
         }
       } else {
+        RopeBase rn = rb;
+        if (rope && col0 < col1) rope_base(col0, rb);
 #pragma unroll 1
         for (int c0 = col0; c0 < col1; c0 += 16) {
           ptx::tmem_ld_32x16(t_lane + c0, a0);
           ptx::tmem_ld_32x16(t_lane + 256 + c0, a1);
-          if (rope) rope_base(c0, rb);
+          if (rope && c0 + 16 < col1) rope_base(c0 + 16, rn);   // one chunk ahead
           ptx::tmem_ld_wait();
           chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
+          rb.c = rn.c; rb.s = rn.s;
           DC_ETRACE(c0)
         }
       }
