@@ -54,7 +54,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const __grid_constant__ CUtensorMap map_vt, const __grid_constant__ CUtensorMap map_kc,
           const __grid_constant__ CUtensorMap map_vc, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t q_full, kv_full[2], kv_empty[2], s_full[2], s_empty[2], p_full[2], pv_done;
+  __shared__ uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], pv_done;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float xchg[2][128];   // row maximum / row sum of each key half
@@ -77,7 +77,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     abort_flag = 0;
     ptx::mbar_init(&q_full, 1);
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(&kv_full[i], 1); ptx::mbar_init(&kv_empty[i], 1);
+      ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1);
+      ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1);
       ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], 256);
       ptx::mbar_init(&p_full[i], 256);
     }
@@ -94,45 +95,63 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const uint32_t tmem_base = tmem_base_s;
 
   if (warp == 0) {
+    // Two producer lanes with a ring of their own each: a K slot is free again as soon as
+    // S = Q K^T of its tile has been computed, a V^T slot only after P V, a softmax later.  With
+    // one ring for both, the load of tile t+2 could not start before P V of tile t and its
+    // latency sat in the loop (2 us per tile); now K runs ahead of V.
+    // Context tiles are also prefetched into L2 kAttnPrefetch tiles ahead (the active tiles were
+    // just written: L2-resident).
     if (lane == 0) {
       ptx::mbar_expect_tx(&q_full, 2 * kSub);
       ptx::tma_load_2d(Qs, &map_q, &q_full, h * kHd, row0 + qt * 128);
       ptx::tma_load_2d(Qs + kSub, &map_q, &q_full, h * kHd + 64, row0 + qt * 128);
-      // With two stages a tile's load can only be issued when the tile two before it has been
-      // consumed, so its full latency sits in the loop; context tiles are therefore prefetched
-      // into L2 kAttnPrefetch tiles ahead (the active tiles were just written: L2-resident).
-      auto prefetch_ctx = [&](int t) {
+      auto prefetch_k = [&](int t) {
         if (t < Tc) {
-          const int j0 = t * kBK;
-          const int krow = (b * p.nkv + g) * p.max_ctx + j0, vrow = (b * p.nkv + g) * kHd;
+          const int krow = (b * p.nkv + g) * p.max_ctx + t * kBK;
           ptx::tma_prefetch_l2_3d(&map_kc, 0, krow, p.layer);
           ptx::tma_prefetch_l2_3d(&map_kc, 64, krow, p.layer);
+        }
+      };
+      for (int t = 2; t < 2 + kAttnPrefetch; ++t) prefetch_k(t);
+      for (int t = 0; t < T; ++t) {
+        const int s = t & 1;
+        prefetch_k(t + 2 + kAttnPrefetch);
+        if (!ptx::mbar_wait(&k_empty[s], (((uint32_t)t >> 1) & 1u) ^ 1u, &abort_flag)) break;
+        uint8_t* Ks = KVs + (size_t)s * 4 * kSub;
+        ptx::mbar_expect_tx(&k_full[s], 2 * kSub);
+        if (t < Tc) {
+          const int krow = (b * p.nkv + g) * p.max_ctx + t * kBK;
+          ptx::tma_load_3d(Ks, &map_kc, &k_full[s], 0, krow, p.layer);
+          ptx::tma_load_3d(Ks + kSub, &map_kc, &k_full[s], 64, krow, p.layer);
+        } else {
+          const int j0 = (t - Tc) * kBK;
+          ptx::tma_load_2d(Ks, &map_k, &k_full[s], g * kHd, row0 + j0);
+          ptx::tma_load_2d(Ks + kSub, &map_k, &k_full[s], g * kHd + 64, row0 + j0);
+        }
+      }
+    } else if (lane == 1) {
+      auto prefetch_v = [&](int t) {
+        if (t < Tc) {
+          const int j0 = t * kBK, vrow = (b * p.nkv + g) * kHd;
           ptx::tma_prefetch_l2_3d(&map_vc, j0, vrow, p.layer);
           ptx::tma_prefetch_l2_3d(&map_vc, j0 + 64, vrow, p.layer);
         }
       };
-      for (int t = 2; t < 2 + kAttnPrefetch; ++t) prefetch_ctx(t);
+      for (int t = 2; t < 2 + kAttnPrefetch; ++t) prefetch_v(t);
       for (int t = 0; t < T; ++t) {
         const int s = t & 1;
-        prefetch_ctx(t + 2 + kAttnPrefetch);
-        if (!ptx::mbar_wait(&kv_empty[s], (((uint32_t)t >> 1) & 1u) ^ 1u, &abort_flag)) break;
-        uint8_t* Ks = KVs + (size_t)s * 4 * kSub;
-        uint8_t* Vs = Ks + 2 * kSub;
-        ptx::mbar_expect_tx(&kv_full[s], 4 * kSub);
+        prefetch_v(t + 2 + kAttnPrefetch);
+        if (!ptx::mbar_wait(&v_empty[s], (((uint32_t)t >> 1) & 1u) ^ 1u, &abort_flag)) break;
+        uint8_t* Vs = KVs + (size_t)s * 4 * kSub + 2 * kSub;
+        ptx::mbar_expect_tx(&v_full[s], 2 * kSub);
         if (t < Tc) {
-          const int j0 = t * kBK;
-          const int krow = (b * p.nkv + g) * p.max_ctx + j0;
-          ptx::tma_load_3d(Ks, &map_kc, &kv_full[s], 0, krow, p.layer);
-          ptx::tma_load_3d(Ks + kSub, &map_kc, &kv_full[s], 64, krow, p.layer);
-          const int vrow = (b * p.nkv + g) * kHd;
-          ptx::tma_load_3d(Vs, &map_vc, &kv_full[s], j0, vrow, p.layer);
-          ptx::tma_load_3d(Vs + kSub, &map_vc, &kv_full[s], j0 + 64, vrow, p.layer);
+          const int j0 = t * kBK, vrow = (b * p.nkv + g) * kHd;
+          ptx::tma_load_3d(Vs, &map_vc, &v_full[s], j0, vrow, p.layer);
+          ptx::tma_load_3d(Vs + kSub, &map_vc, &v_full[s], j0 + 64, vrow, p.layer);
         } else {
           const int j0 = (t - Tc) * kBK;
-          ptx::tma_load_2d(Ks, &map_k, &kv_full[s], g * kHd, row0 + j0);
-          ptx::tma_load_2d(Ks + kSub, &map_k, &kv_full[s], g * kHd + 64, row0 + j0);
-          ptx::tma_load_2d(Vs, &map_vt, &kv_full[s], row0 + j0, g * kHd);
-          ptx::tma_load_2d(Vs + kSub, &map_vt, &kv_full[s], row0 + j0 + 64, g * kHd);
+          ptx::tma_load_2d(Vs, &map_vt, &v_full[s], row0 + j0, g * kHd);
+          ptx::tma_load_2d(Vs + kSub, &map_vt, &v_full[s], row0 + j0 + 64, g * kHd);
         }
       }
     }
@@ -146,7 +165,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       const uint64_t dk0 = hi | (uint64_t)(ptx::smem_u32(KVs) >> 4);                 // stage 0; stage 1 = + 4*kSub
       const uint64_t dv0 = dk0 + (2 * kSub >> 4);
       const uint64_t dp0 = hi | (uint64_t)(ptx::smem_u32(Ps) >> 4);                  // buffer 0; buffer 1 = + 2*kSub
-      const uint32_t b_kv_full = ptx::smem_u32(&kv_full[0]), b_kv_empty = ptx::smem_u32(&kv_empty[0]);
+      const uint32_t b_k_full = ptx::smem_u32(&k_full[0]), b_k_empty = ptx::smem_u32(&k_empty[0]);
+      const uint32_t b_v_full = ptx::smem_u32(&v_full[0]), b_v_empty = ptx::smem_u32(&v_empty[0]);
       const uint32_t b_s_full = ptx::smem_u32(&s_full[0]), b_s_empty = ptx::smem_u32(&s_empty[0]);
       const uint32_t b_p_full = ptx::smem_u32(&p_full[0]), b_pv_done = ptx::smem_u32(&pv_done);
       constexpr uint64_t kSubU = kSub >> 4;   // one 64-column sub-tile in descriptor units
@@ -154,7 +174,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       auto issue_qk = [&](int t) {
         const uint32_t s = (uint32_t)t & 1u;
         const uint32_t ph = ((uint32_t)t >> 1) & 1u;
-        if (!ptx::mbar_wait_a(b_kv_full + 8u * s, ph, &abort_flag)) return false;
+        if (!ptx::mbar_wait_a(b_k_full + 8u * s, ph, &abort_flag)) return false;
         if (!ptx::mbar_wait_a(b_s_empty + 8u * s, ph ^ 1u, &abort_flag)) return false;
         ptx::tc_fence_after();
         const uint64_t dk = dk0 + s * (4 * kSubU);
@@ -166,10 +186,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           ptx::umma_bf16_acc(d, dq + off, dk + off, idesc);
         }
         ptx::umma_commit_a(b_s_full + 8u * s);
+        ptx::umma_commit_a(b_k_empty + 8u * s);   // the K slot is free once S is there
         return true;
       };
       auto issue_pv = [&](int t) {
         const uint32_t s = (uint32_t)t & 1u;
+        if (!ptx::mbar_wait_a(b_v_full + 8u * s, ((uint32_t)t >> 1) & 1u, &abort_flag)) return false;
         if (!ptx::mbar_wait_a(b_p_full + 8u * s, ((uint32_t)t >> 1) & 1u, &abort_flag)) return false;
         ptx::tc_fence_after();
         const uint64_t dp = dp0 + s * (2 * kSubU);
@@ -182,7 +204,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           ptx::umma_bf16_acc(d, dp + off, dv + off, idesc);
         }
         ptx::umma_commit_a(b_pv_done);
-        ptx::umma_commit_a(b_kv_empty + 8u * s);
+        ptx::umma_commit_a(b_v_empty + 8u * s);
         return true;
       };
       if (ok && T > 0) ok = issue_qk(0);
@@ -221,9 +243,23 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         ptx::mbar_arrive(&s_empty[s]);
+        // The softmax warps are bound by instruction issue (85% of the issue slots of their
+        // schedulers), so the per-element work is kept to max, fma, ex2, add and half a convert:
+        // keys beyond the valid length are set to -inf once (only the last tile of a kind has
+        // any; whatever the cache holds there, NaN included, is overwritten), after which they
+        // need no further test (ex2(-inf) = 0); maxima and sums run in four independent chains.
+        if (vloc < 64) {
 #pragma unroll
-        for (int j = 0; j < 64; ++j)
-          if (j < vloc) mx = fmaxf(mx, sv[j]);
+          for (int j = 0; j < 64; ++j)
+            if (j >= vloc) sv[j] = -INFINITY;
+        }
+        float m0 = sv[0], m1 = sv[1], m2 = sv[2], m3 = sv[3];
+#pragma unroll
+        for (int j = 4; j < 64; j += 4) {
+          m0 = fmaxf(m0, sv[j]); m1 = fmaxf(m1, sv[j + 1]);
+          m2 = fmaxf(m2, sv[j + 2]); m3 = fmaxf(m3, sv[j + 3]);
+        }
+        mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
       }
       xchg[half][r] = mx;
       pair_sync();
@@ -235,7 +271,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       const bool raise = m_tile > m_run + kRescaleGap;   // true on the first tile (m_run = -inf)
       const float m_new = raise ? m_tile : m_run;
       const float alpha = raise ? attn_ex2(m_run - m_new) : 1.f;  // 0 on the first tile
-      float l_tile = 0.f;
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      const float scale = p.scale_log2, neg_m = -m_new;
       // keys [kbase, kbase+64) are sub-tile `half` of the P buffer: 8 chunks of 8 keys per row
       uint8_t* prow = Ps + (size_t)s * 2 * kSub + half * kSub + r * 128;
 #pragma unroll
@@ -244,9 +281,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
           const int k0 = c * 32 + j;
-          const float p0 = (k0 < vloc) ? attn_ex2(fmaf(sv[k0], p.scale_log2, -m_new)) : 0.f;
-          const float p1 = (k0 + 1 < vloc) ? attn_ex2(fmaf(sv[k0 + 1], p.scale_log2, -m_new)) : 0.f;
-          l_tile += p0 + p1;
+          const float p0 = attn_ex2(fmaf(sv[k0], scale, neg_m));
+          const float p1 = attn_ex2(fmaf(sv[k0 + 1], scale, neg_m));
+          if ((j & 6) == 0) l0 += p0 + p1;
+          else if ((j & 6) == 2) l1 += p0 + p1;
+          else if ((j & 6) == 4) l2 += p0 + p1;
+          else l3 += p0 + p1;
           __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
           packed[j >> 1] = *reinterpret_cast<uint32_t*>(&pr);
         }
@@ -257,11 +297,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
               make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
         }
       }
-      l_run = l_run * alpha + l_tile;
+      l_run = l_run * alpha + ((l0 + l1) + (l2 + l3));
       m_run = m_new;
       if (is_ctx && valid < kBK) {
         // cached keys beyond ctx_len: zero the V^T columns so that 0 * garbage cannot make NaN
-        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&kv_full[s], ph, &abort_flag));
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&v_full[s], ph, &abort_flag));
         if (ok) {
           uint8_t* vrow = KVs + (size_t)s * 4 * kSub + 2 * kSub + half * kSub + r * 128;
           for (int cc = vloc; cc < 64; ++cc)
