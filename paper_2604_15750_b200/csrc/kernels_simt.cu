@@ -513,8 +513,11 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
   const T* wr = lm_head + (size_t)tok * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) wrow[i] = to_f<T>(wr[i]);
   __syncthreads();
+  // one window position per warp: blockIdx.z picks the group of positions, so that a step's W * W
+  // dot products are spread over W * W / 8 CTAs instead of W (the kernel is bound by the latency
+  // of a row load, not by bytes: 37 -> 8 us at W = 64)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  for (int i = warp; i < W; i += nw) {
+  for (int i = blockIdx.z * nw + warp; i < W; i += gridDim.z * nw) {
     const T* hr = h + (size_t)lm_row(m, 0, b * m.W_cap + i) * d;
     float acc = 0.f;
     // d is a multiple of 4: four elements per lane and step (8- or 16-byte loads), eight steps
@@ -547,7 +550,7 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
 template <typename T>
 void launch_xlogp(const T* h, const T* lm_head, const int32_t* ws_pred, const float* ws_lse, int d,
                   const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s) {
-  dim3 grid(m.W_cap, m.batch);
+  dim3 grid(m.W_cap, m.batch, (m.W_cap + 7) / 8);
   k_xlogp<T><<<grid, 256, d * sizeof(float), s>>>(h, lm_head, ws_pred, ws_lse, d, m, max_window,
                                                   xlogp);
 }
