@@ -225,6 +225,27 @@ DC_API int dc_select(dc_ctx* ctx, const dc_select_in* in, const dc_select_out* o
 /* ---- the decoding loop around the step (Section 3, Eq. 1-2; Section 4.2 "starting from the
  * current frontier ...") ---------------------------------------------------------------------- */
 
+/* Prefill: the K / V of n_ids[b] clean tokens per sequence (a prompt, or any run of decoded
+ * tokens whose cache is to be rebuilt), computed by one bidirectional pass over those tokens - they
+ * attend one another and the ctx_len[b] keys already in the cache (Section 3: the DLM attends the
+ * whole known sequence; Section 4.1 / "compatible with existing block-wise cache techniques") -
+ * and written into the caches at keys ctx_len[b] .. ctx_len[b] + n_ids[b] - 1, every layer.  The
+ * same kernels as dc_step without window rows; no LM head.  A prompt goes through in one call
+ * (the pass is bidirectional, so chunks would not see each other): n_ids[b] <= max_last and
+ * ctx_len[b] + n_ids[b] <= max_ctx, DC_ERR_SHAPE otherwise.  Asynchronous on the handle's stream. */
+typedef struct dc_prefill_in {
+  int32_t batch;
+  void* k_cache;             /* device, layouts as in dc_step, written                        */
+  void* v_cache;             /* device, written                                               */
+  const int32_t* ctx_len;    /* host [batch], may be null (all 0)                             */
+  const int32_t* ids;        /* device [batch][max_last]                                      */
+  const int32_t* n_ids;      /* host [batch]                                                  */
+} dc_prefill_in;
+typedef struct dc_prefill_out {
+  int32_t* status;           /* device [batch]                                                */
+} dc_prefill_out;
+DC_API int dc_prefill(dc_ctx* ctx, const dc_prefill_in* in, const dc_prefill_out* out);
+
 /* Eq. (2): y_i <- yhat_i for the selected, still masked positions of the current block
  * window[0, block_len); remaining[b] = masked positions left in that block. */
 typedef struct dc_commit_in {

@@ -208,6 +208,22 @@ def forward(cfg: OracleConfig, w: OracleWeights, tok: np.ndarray, pos0: int,
     return x
 
 
+def prefill(cfg: OracleConfig, w: OracleWeights, ids: np.ndarray, k_ctx=None, v_ctx=None,
+            ctx_len: int = 0, n_layers: int | None = None):
+    """K / V of a run of clean tokens (a prompt), as one bidirectional pass over them makes
+    them: the tokens sit at positions ctx_len + r, attend one another and the ctx_len cached
+    keys (Section 3: the model attends the whole known sequence, no causal mask).
+    Returns (k, v), each [n_layers, n_kv_heads, len(ids), head_dim], K rotated.
+    """
+    if k_ctx is not None:
+        k_ctx, v_ctx = k_ctx[:, :, :ctx_len, :], v_ctx[:, :, :ctx_len, :]
+    _, kv = forward(cfg, w, np.asarray(ids), int(ctx_len), k_ctx, v_ctx, return_kv=True,
+                    n_layers=n_layers)
+    k = np.stack([np.transpose(k_, (1, 0, 2)) for k_, _ in kv])
+    v = np.stack([np.transpose(v_, (1, 0, 2)) for _, v_ in kv])
+    return k, v
+
+
 def final_hidden(cfg: OracleConfig, w: OracleWeights, x_rows: np.ndarray) -> np.ndarray:
     """LM-head input: final RMSNorm of the given rows (rounded when the path is bf16)."""
     return _gemm_in(rmsnorm(x_rows, w.final_norm, cfg.rms_eps), cfg)

@@ -19,7 +19,7 @@ DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
                "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
-           "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate"]
+           "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate", "dc_prefill"]
 
 
 class DepCapError(RuntimeError):
@@ -86,6 +86,15 @@ class dc_select_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("sel_mask", "sel_idx", "sel_count")]
 
 
+class dc_prefill_in(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("ctx_len", _I32P), ("ids", C.c_void_p), ("n_ids", _I32P)]
+
+
+class dc_prefill_out(C.Structure):
+    _fields_ = [("status", C.c_void_p)]
+
+
 class dc_commit_in(C.Structure):
     _fields_ = [("batch", C.c_int32), ("win_ids", C.c_void_p), ("pred_id", C.c_void_p),
                 ("sel_mask", C.c_void_p), ("block_len", C.c_void_p), ("win_len", _I32P)]
@@ -139,6 +148,7 @@ def load_library(path: str | None = None):
     lib_.dc_select.argtypes = [C.c_void_p, C.POINTER(dc_select_in), C.POINTER(dc_select_out)]
     lib_.dc_signals_static.argtypes = [C.POINTER(dc_signals_in), C.POINTER(dc_signals_out),
                                        C.c_void_p]
+    lib_.dc_prefill.argtypes = [C.c_void_p, C.POINTER(dc_prefill_in), C.POINTER(dc_prefill_out)]
     lib_.dc_commit.argtypes = [C.c_void_p, C.POINTER(dc_commit_in), C.POINTER(dc_commit_out)]
     lib_.dc_generate.argtypes = [C.c_void_p, C.POINTER(dc_generate_in),
                                  C.POINTER(dc_generate_out)]
@@ -364,6 +374,19 @@ class DepCap:
         so = dc_select_out(**{k: _ptr(v) for k, v in self.sel.items()})
         self._check(self._lib.dc_select(self._ctx, C.byref(si), C.byref(so)))
         return self.sel
+
+    def prefill(self, k_cache, v_cache, ids, n_ids, ctx_len=None):
+        """K / V of n_ids[b] clean tokens (device ids [B, max_last]) into the caches at keys
+        ctx_len[b] ...; returns the device status tensor."""
+        B = len(n_ids)
+        n_ = _host_i32(n_ids, B)
+        c_ = _host_i32(ctx_len if ctx_len is not None else [0] * B, B)
+        self._keep_pf = (k_cache, v_cache, ids, n_, c_)
+        pi = dc_prefill_in(batch=B, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                           ctx_len=C.cast(c_, _I32P), ids=_ptr(ids), n_ids=C.cast(n_, _I32P))
+        po = dc_prefill_out(status=_ptr(self.out["status"]))
+        self._check(self._lib.dc_prefill(self._ctx, C.byref(pi), C.byref(po)))
+        return self.out["status"]
 
     def commit(self, win_ids, win_len, pred_id=None, sel_mask=None, block_len=None):
         """Eq. (2) in place on win_ids; returns the device tensor of masked positions left."""

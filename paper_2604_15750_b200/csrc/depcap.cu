@@ -124,7 +124,8 @@ T* ws_alloc(dc_ctx* c, size_t n, bool* ok) {
 }
 
 int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const int32_t* last_len,
-               const int32_t* win_len, const int32_t* remain_len, SeqMeta* m) {
+               const int32_t* win_len, const int32_t* remain_len, SeqMeta* m,
+               bool no_window = false) {
   const dc_config& g = c->cfg;
   if (batch < 1 || batch > g.max_batch)
     return fail(c, DC_ERR_SHAPE, "batch %d outside [1, max_batch=%d]", batch, g.max_batch);
@@ -133,12 +134,13 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
   m->nv = (flags & DC_STEP_INFLUENCE) ? 2 : 1;
   int maxR = 0, maxW = 0;
   for (int b = 0; b < batch; ++b) {
-    const int P = ctx_len ? ctx_len[b] : 0, Lb = last_len ? last_len[b] : 0, W = win_len[b];
+    const int P = ctx_len ? ctx_len[b] : 0, Lb = last_len ? last_len[b] : 0;
+    const int W = no_window ? 0 : win_len[b];
     if (P < 0 || P > g.max_ctx)
       return fail(c, DC_ERR_SHAPE, "ctx_len[%d]=%d outside [0, max_ctx=%d]", b, P, g.max_ctx);
     if (Lb < 0 || Lb > g.max_last)
       return fail(c, DC_ERR_SHAPE, "last_len[%d]=%d outside [0, max_last=%d]", b, Lb, g.max_last);
-    if (W < 1 || W > g.max_window)
+    if (!no_window && (W < 1 || W > g.max_window))
       return fail(c, DC_ERR_SHAPE, "win_len[%d]=%d outside [1, max_window=%d]", b, W,
                   g.max_window);
     m->ctx_len[b] = P; m->last_len[b] = Lb; m->win_len[b] = W;
@@ -152,6 +154,7 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
   const int npos = batch * m->W_cap;
   const int gmax = 128 / m->nv;  // an LM-head group is [G curr rows ; G prev rows] <= 128 rows
   m->G = npos < gmax ? npos : gmax;
+  if (m->G < 1) m->G = 1;   // no window rows (prefill): the LM head does not run
   m->npos_pad = round_up(npos, m->G);
   return DC_OK;
 }
@@ -165,7 +168,8 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
   } while (0)
 
 template <typename T>
-int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqMeta& m) {
+int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqMeta& m,
+             const bool kv_only = false) {
   const dc_config& g = c->cfg;
   cudaStream_t s = c->stream;
   Profiler& pf = c->prof;
@@ -204,6 +208,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     if (rc != DC_OK) return fail(c, rc, "dense chain failed: %s", tc_error(c->tc));
     for (int l = 0; l < L; ++l) {
       if (export_kv) tc_export_kv(c->tc, l, m, (__nv_bfloat16*)in->k_cache, (__nv_bfloat16*)in->v_cache);
+      if (kv_only && l + 1 == L) break;   // prefill: nothing after the last layer's K / V is used
       pf.begin(DC_STAGE_ATTN, 1);
       rc = tc_attention(c->tc, l, m, (const __nv_bfloat16*)in->k_cache,
                         (const __nv_bfloat16*)in->v_cache);
@@ -232,7 +237,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
       int rc = tc_layer(c->tc, l, m, c->x, (const __nv_bfloat16*)a,
                         (const __nv_bfloat16*)in->k_cache, (const __nv_bfloat16*)in->v_cache,
                         c->cos_sin, (const __nv_bfloat16*)c->norm2[l],
-                        &part, &nsplit, &part_stride, pf, export_kv);
+                        &part, &nsplit, &part_stride, pf, export_kv, kv_only && l + 1 == g.n_layers);
       if (rc != DC_OK) return fail(c, rc, "tensor-core layer %d failed: %s", l, tc_error(c->tc));
       continue;
     }
@@ -247,6 +252,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     if (export_kv)
       launch_export_kv<T>(k, v, 0, m, nkv, hd, g.max_ctx, (T*)in->k_cache + (size_t)l * k_layer,
                           (T*)in->v_cache + (size_t)l * k_layer, s);
+    if (kv_only && l + 1 == g.n_layers) break;
     pf.begin(DC_STAGE_ATTN, 1);
     launch_attn_simt<T>(q, k, v, kc, vc, g.max_ctx, m, nq, nkv, hd, o, s);
     pf.end();
@@ -267,6 +273,11 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     DC_CHECK_LAUNCH(c);
   }
 
+  if (kv_only) {
+    if (c->use_tc) tc_flush_status(c->tc, out->status, m.batch);
+    DC_CHECK_LAUNCH(c);
+    return DC_OK;
+  }
   pf.begin(DC_STAGE_NORM, in->h_final_in ? 2 : 1);
   launch_final_norm<T>(c->x, part, nsplit, part_stride, (const T*)c->final_norm, g.rms_eps, d, m,
                        h, s);
@@ -531,6 +542,35 @@ int dc_select(dc_ctx* c, const dc_select_in* in, const dc_select_out* out) {
                 c->cfg.max_window, out->sel_mask, out->sel_idx, out->sel_count, c->stream);
   DC_CHECK_LAUNCH(c);
   return DC_OK;
+}
+
+int dc_prefill(dc_ctx* c, const dc_prefill_in* in, const dc_prefill_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!in || !out || !in->ids || !in->n_ids || !in->k_cache || !in->v_cache || !out->status)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument");
+  SeqMeta m;
+  int rc = build_meta(c, in->batch, 0, in->ctx_len, in->n_ids, nullptr, nullptr, &m, true);
+  if (rc != DC_OK) return rc;
+  for (int b = 0; b < m.batch; ++b) {
+    if (m.last_len[b] < 1) return fail(c, DC_ERR_SHAPE, "n_ids[%d] must be positive", b);
+    if (m.ctx_len[b] + m.last_len[b] > c->cfg.max_ctx)
+      return fail(c, DC_ERR_SHAPE, "ctx_len[%d] + n_ids[%d] = %d exceeds max_ctx=%d", b, b,
+                  m.ctx_len[b] + m.last_len[b], c->cfg.max_ctx);
+  }
+  dc_step_in si{};
+  si.batch = in->batch; si.flags = DC_STEP_EXPORT_KV;
+  si.k_cache = in->k_cache; si.v_cache = in->v_cache; si.ctx_len = in->ctx_len;
+  si.last_ids = in->ids; si.last_len = in->n_ids;
+  si.win_ids = c->g_win;       // never read: no sequence has window rows
+  dc_step_out so{};
+  so.status = out->status;
+  int dev = -1;
+  cudaGetDevice(&dev);
+  if (dev != c->device) cudaSetDevice(c->device);
+  c->prof.reset(false, c->stream);
+  rc = c->bf16 ? run_step<__nv_bfloat16>(c, &si, &so, m, true) : run_step<float>(c, &si, &so, m, true);
+  if (dev != c->device && dev >= 0) cudaSetDevice(dev);
+  return rc;
 }
 
 int dc_commit(dc_ctx* c, const dc_commit_in* in, const dc_commit_out* out) {

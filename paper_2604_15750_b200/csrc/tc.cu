@@ -478,7 +478,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
-             StageHook& hook, bool export_kv) {
+             StageHook& hook, bool export_kv, bool kv_only) {
   const dc_config& g = t->g;
   const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
   const int M = m.nv * m.batch * m.R_cap;
@@ -501,6 +501,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 
   if (export_kv)
     tc_export_kv(t, layer, m, const_cast<__nv_bfloat16*>(k_cache), const_cast<__nv_bfloat16*>(v_cache));
+  if (kv_only) return DC_OK;   // prefill, last layer: only its K / V were wanted
   hook.begin(DC_STAGE_ATTN, 1);
   rc = tc_attention(t, layer, m, k_cache, v_cache);
   hook.end();

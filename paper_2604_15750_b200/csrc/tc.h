@@ -41,7 +41,7 @@ const char* tc_error(const TcState* t);
 int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloat16* a,
              const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, const float* cos_sin,
              const __nv_bfloat16* norm2, const float** part, int* nsplit, size_t* part_stride,
-             StageHook& hook, bool export_kv = false);
+             StageHook& hook, bool export_kv = false, bool kv_only = false);
 
 // Attention of one layer alone (reads the rotated q / k / transposed v the QKV epilogue wrote).
 int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,

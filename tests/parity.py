@@ -34,10 +34,7 @@ def oracle_cfg(wl, hyper: Hyper, n_layers=None):
 
 def oracle_prefix_kv(ocfg, ow, prompt_ids):
     """Context cache made by the oracle's own forward over the prompt alone (bidirectional)."""
-    _, kv = O.forward(ocfg, ow, np.asarray(prompt_ids), 0, None, None, return_kv=True)
-    k = np.stack([np.transpose(k_, (1, 0, 2)) for k_, _ in kv])        # [L, nkv, P, hd]
-    v = np.stack([np.transpose(v_, (1, 0, 2)) for _, v_ in kv])
-    return k, v
+    return O.prefill(ocfg, ow, np.asarray(prompt_ids))
 
 
 class Case:
