@@ -222,6 +222,80 @@ def run_reference(args, wl, rank, world):
     print(json.dumps(line))
 
 
+def run_generate(args, wl, dev):
+    """Block-wise generation of --gen-len tokens per sequence behind the workload's context
+    (dc_generate: boundary step + denoising steps per block, host read-back every step)."""
+    import time
+    from paper_2604_15750_b200 import DepCap, pack_kv_cache
+    n_layers = args.layers or wl.n_layers
+    weights = inputs.make_weights(wl, device=dev, n_layers=n_layers)
+    weights["lm_head"] = weights["lm_head"] * args.lm_scale
+    k_log, v_log = inputs.make_ctx_kv(wl, device=dev, n_layers=n_layers)
+    lens = {k: [int(x) for x in v] for k, v in inputs.make_lengths(wl).items()}
+    N = args.gen_len
+    max_ctx = (wl.ctx_max + N + 63) // 64 * 64
+    eng = DepCap.from_workload(wl, weights, n_layers=n_layers, max_ctx=max_ctx,
+                               max_last=max(wl.win_len, 16), max_window=(wl.win_len + 15) // 16 * 16)
+    kc, vc = pack_kv_cache(k_log, v_log, eng.max_batch, eng.max_ctx)
+    eng.generate(kc, vc, lens["ctx_len"], min(N, 32))           # warm-up
+    eng.synchronize()
+    t0 = time.perf_counter()
+    tok, blocks, nfe = eng.generate(kc, vc, lens["ctx_len"], N)
+    eng.synchronize()
+    dt = time.perf_counter() - t0
+    nb = [len(b) for b in blocks]
+    print(json.dumps(dict(metric="generated_tokens_per_s", value=wl.batch * N / dt, unit="tokens/s",
+                          n_gpus=1, mode="generate", ms=dt * 1e3, nfe=nfe,
+                          tokens_per_forward=wl.batch * N / nfe, ms_per_forward=dt * 1e3 / nfe,
+                          blocks_per_sequence=nb, mean_block_len=float(N * wl.batch / max(sum(nb), 1)),
+                          dtype="bf16" if wl.dtype == "bf16" else "f32", data="synthetic",
+                          config=dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, gen_len=N,
+                                      layers=n_layers, lm_head_scale=args.lm_scale,
+                                      timing="wall clock around dc_generate, host read-back every step"))),
+          flush=True)
+    eng.close()
+
+
+def run_prefill(args, wl, dev):
+    """dc_prefill of --prompt-len tokens per sequence (one bidirectional pass, K / V export)."""
+    from paper_2604_15750_b200 import DepCap
+    n_layers = args.layers or wl.n_layers
+    weights = inputs.make_weights(wl, device=dev, n_layers=n_layers)
+    P = args.prompt_len
+    max_ctx = (P + 63) // 64 * 64
+    eng = DepCap.from_workload(wl, weights, n_layers=n_layers, max_ctx=max_ctx, max_last=P,
+                               max_window=16)
+    B, nkv, hd = wl.batch, wl.n_kv_heads, wl.head_dim
+    kc = torch.zeros((n_layers, B, nkv, max_ctx, hd), dtype=wl.torch_dtype, device=dev)
+    vc = torch.zeros((n_layers, B, nkv, hd, max_ctx), dtype=wl.torch_dtype, device=dev)
+    g = torch.Generator().manual_seed(wl.seed)
+    ids = torch.randint(0, wl.vocab - 1, (B, P), dtype=torch.int32, generator=g).to(dev)
+    for _ in range(args.warmup):
+        eng.prefill(kc, vc, ids, [P] * B)
+    eng.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = min(args.steps, 20)
+    e0.record(eng.stream)
+    for _ in range(steps):
+        eng.prefill(kc, vc, ids, [P] * B)
+    e1.record(eng.stream)
+    eng.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    # all layers but the last run in full; the last stops after its QKV projection
+    qkv = wl.d_model * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim
+    flops = 2.0 * B * P * ((n_layers - 1) * _layer_param_count(wl) + qkv)
+    flops += 4.0 * B * (n_layers - 1) * wl.n_q_heads * wl.head_dim * P * P      # attention
+    peaks = _peaks()
+    print(json.dumps(dict(metric="prefill_tokens_per_s", value=B * P / (ms * 1e-3), unit="tokens/s",
+                          n_gpus=1, mode="prefill", ms=ms, tflops=flops / (ms * 1e-3) / 1e12,
+                          frac_of_bf16_peak=flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+                          peak_source=peaks["source"], dtype="bf16" if wl.dtype == "bf16" else "f32",
+                          data="synthetic",
+                          config=dict(workload=wl.name, batch=B, prompt_len=P, layers=n_layers))),
+          flush=True)
+    eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -232,6 +306,13 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debug: run fewer layers (invalid as a result)")
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="step", choices=["step", "generate", "prefill"],
+                    help="step: the bench line; generate / prefill: measurements of the decoding "
+                         "loop and of dc_prefill on the same model shape (one GPU, own JSON line)")
+    ap.add_argument("--gen-len", type=int, default=256)
+    ap.add_argument("--prompt-len", type=int, default=1024)
+    ap.add_argument("--lm-scale", type=float, default=8.0,
+                    help="generate: factor on the random-init LM head so that predictions are peaked")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", "0"))
@@ -248,6 +329,10 @@ def main():
     assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU path"
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if args.mode != "step":
+        if rank == 0:
+            (run_generate if args.mode == "generate" else run_prefill)(args, wl, dev)
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist
