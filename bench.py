@@ -309,6 +309,9 @@ def main():
     ap.add_argument("--mode", default="step", choices=["step", "generate", "prefill"],
                     help="step: the bench line; generate / prefill: measurements of the decoding "
                          "loop and of dc_prefill on the same model shape (one GPU, own JSON line)")
+    ap.add_argument("--prev", default="recomputed", choices=["recomputed", "carried"],
+                    help="step mode: p_prev from a second variant in the pass (the bench line) or from "
+                         "rows carried in (DC_STEP_CARRIED_PREV: half the rows through the stack)")
     ap.add_argument("--gen-len", type=int, default=256)
     ap.add_argument("--prompt-len", type=int, default=1024)
     ap.add_argument("--lm-scale", type=float, default=8.0,
@@ -356,6 +359,8 @@ def main():
     last_d, win_d, hf_d = last_h.to(dev), win_h.to(dev), hf_h.to(dev)
     step_kw = dict(k_cache=kc, v_cache=vc, ctx_len=lens["ctx_len"], last_len=lens["last_len"],
                    win_len=lens["win_len"], remain_len=lens["remain_len"])
+    if args.prev == "carried":
+        step_kw["carried"] = (hf_d[:, 1].contiguous(), lens["win_len"])
     stream = eng.stream
 
     def one_step():
@@ -478,6 +483,7 @@ def main():
                 scaling="weak", vs_baseline=None, dtype="bf16" if wl.dtype == "bf16" else "f32",
                 data="synthetic",
                 config=_config(wl, n_layers, committed_per_step=committed, kernels=args.kernels,
+                               **({"variants": "curr + carried prev rows"} if args.prev == "carried" else {}),
                                status=status_bad),
                 clocks=clocks,
                 e2e=dict(value=committed_e2e / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,

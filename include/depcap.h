@@ -71,6 +71,12 @@ enum { DC_MAX_BATCH = 32, DC_MAX_WINDOW = 256 };
 enum {
   DC_STEP_INFLUENCE = 1, /* also run the prev variant and reduce I_k (Eq. 3)                */
   DC_STEP_BOUNDARY = 2,  /* run the boundary rule (Section 4.2) and write block_len         */
+  DC_STEP_CARRIED_PREV = 8, /* p_prev comes from rows the caller carried over from an earlier step
+                            (h_prev_in, prev_len) instead of a second variant in this pass: the
+                            stack runs the curr rows only (half the rows).  This is how the
+                            paper's own implementation obtains the two distributions ("logits
+                            immediately before and after decoding B", Implementation
+                            Approximation).  Not together with DC_STEP_INFLUENCE              */
   DC_STEP_EXPORT_KV = 4  /* append the last decoded block's K / V (curr variant, every layer) to
                             the caches at keys ctx_len[b] .. ctx_len[b] + last_len[b] - 1: the
                             library WRITES k_cache / v_cache there (block-wise cache reuse,
@@ -142,6 +148,13 @@ typedef struct dc_step_in {
    * stack's output as the LM-head input (the stack still runs).  For tests and benchmarks that
    * need shaped distributions from random-init weights.  Null in normal use. */
   const void* h_final_in;
+  /* DC_STEP_CARRIED_PREV: device [batch][max_window][d_model], model dtype: row k of sequence b is
+   * the LM-head input (final-normed hidden state, as h_out of an earlier step gives it) whose
+   * distribution serves as p_prev of window position k, for k < prev_len[b] (host [batch],
+   * 0..win_len[b]).  Positions k >= prev_len[b] have no earlier prediction: I_k = 0 there, so the
+   * boundary rule ends the block at prev_len[b] at the latest; prev_len[b] = 0 is a cold start. */
+  const void* h_prev_in;
+  const int32_t* prev_len;
 } dc_step_in;
 
 /* Caller-owned device buffers; rows b >= batch and columns k >= win_len[b] are not written.
@@ -158,6 +171,9 @@ typedef struct dc_step_out {
   float* cum_score;     /* [batch][max_window] sum_{j<=k} S_j     (DC_STEP_BOUNDARY)        */
   int32_t* block_len;   /* [batch] next block length L            (DC_STEP_BOUNDARY)        */
   int32_t* status;      /* [batch] DC_OK or a device-side dc_status; required               */
+  void* h_out;          /* optional, [batch][max_window][d_model], model dtype: the LM-head input
+                           rows of the curr variant, to be carried into a later step's h_prev_in
+                           (row k of this window is row k - L of the next one after a block of L) */
 } dc_step_out;
 
 typedef struct dc_boundary_in {

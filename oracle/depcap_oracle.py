@@ -397,7 +397,7 @@ def cap_select(conf: np.ndarray, masked: np.ndarray, xlogp: np.ndarray, block_le
 def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
          last_ids: np.ndarray, win_ids: np.ndarray, remain_len: int,
          influence: bool = True, h_final=None, n_layers: int | None = None,
-         return_kv: bool = False) -> dict:
+         return_kv: bool = False, carried=None) -> dict:
     """All per-step outputs for one sequence.
 
     curr variant rows = last decoded block followed by the window; prev variant = the same
@@ -407,6 +407,13 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
     """
     Lb, W = len(last_ids), len(win_ids)
     have_prev = bool(influence and Lb > 0)
+    if carried is not None:
+        # p_prev carried from an earlier pass ("logits immediately before and after decoding B",
+        # Implementation Approximation): carried = (rows [>= prev_len, d], prev_len); row k is the
+        # LM-head input whose distribution is p_prev of window position k.  Positions without a
+        # carried row get p_prev = p_curr, hence I_k = 0.  No second pass runs.
+        influence = False
+        have_prev = False
     if k_ctx is not None:
         k_ctx, v_ctx = k_ctx[:, :, :ctx_len, :], v_ctx[:, :, :ctx_len, :]
     if h_final is None:
@@ -428,6 +435,12 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
         kv_last = None
         h_curr = _gemm_in(h_final[0], cfg)
         h_prev = _gemm_in(h_final[1], cfg) if have_prev else None
+    if carried is not None:
+        rows, n_prev = carried
+        n_prev = int(n_prev)
+        h_prev = np.array(h_curr, dtype=np.float64, copy=True)
+        h_prev[:n_prev] = _gemm_in(np.asarray(rows, dtype=np.float64)[:n_prev], cfg)
+        have_prev = n_prev > 0
     z = logits_of(h_curr, w.lm_head, cfg)
     zp = logits_of(h_prev, w.lm_head, cfg) if have_prev else None
     pred, conf, ent, infl, lse, lse_prev = signals_from_logits(z, zp)

@@ -14,7 +14,7 @@ _LIB_PATH = os.path.join(_HERE, "libdepcap.so")
 
 DC_OK = 0
 DC_F32, DC_BF16 = 0, 1
-DC_STEP_INFLUENCE, DC_STEP_BOUNDARY, DC_STEP_EXPORT_KV = 1, 2, 4
+DC_STEP_INFLUENCE, DC_STEP_BOUNDARY, DC_STEP_EXPORT_KV, DC_STEP_CARRIED_PREV = 1, 2, 4, 8
 DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
                "boundary", "dense"]
@@ -57,13 +57,14 @@ class dc_step_in(C.Structure):
     _fields_ = [("batch", C.c_int32), ("flags", C.c_int32), ("k_cache", C.c_void_p),
                 ("v_cache", C.c_void_p), ("ctx_len", _I32P), ("last_ids", C.c_void_p),
                 ("last_len", _I32P), ("win_ids", C.c_void_p), ("win_len", _I32P),
-                ("remain_len", _I32P), ("h_final_in", C.c_void_p)]
+                ("remain_len", _I32P), ("h_final_in", C.c_void_p), ("h_prev_in", C.c_void_p),
+                ("prev_len", _I32P)]
 
 
 class dc_step_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("pred_id", "conf", "entropy", "influence", "lse", "xlogp", "score",
-                 "cum_influence", "cum_score", "block_len", "status")]
+                 "cum_influence", "cum_score", "block_len", "status", "h_out")]
 
 
 class dc_boundary_in(C.Structure):
@@ -307,12 +308,16 @@ class DepCap:
     # -- dc_step ---------------------------------------------------------------------------
     def _step_structs(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len,
                       remain_len, influence=True, boundary=True, h_final=None, want_xlogp=True,
-                      export_kv=False):
+                      export_kv=False, carried=None, h_out=None):
         B = len(win_len)
         self._keep = (k_cache, v_cache, last_ids, win_ids, h_final,
                       _host_i32(ctx_len, B), _host_i32(last_len, B), _host_i32(win_len, B),
                       _host_i32(remain_len, B))
+        if carried is not None:      # (h_prev_in [B, max_window, d], prev_len): p_prev carried in
+            influence = False
+            self._keep_c = (carried[0], _host_i32(carried[1], B))
         si = dc_step_in(batch=B, flags=(DC_STEP_INFLUENCE if influence else 0) |
+                        (DC_STEP_CARRIED_PREV if carried is not None else 0) |
                         (DC_STEP_BOUNDARY if boundary else 0) |
                         (DC_STEP_EXPORT_KV if export_kv else 0),
                         k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
@@ -320,18 +325,24 @@ class DepCap:
                         last_len=C.cast(self._keep[6], _I32P), win_ids=_ptr(win_ids),
                         win_len=C.cast(self._keep[7], _I32P),
                         remain_len=C.cast(self._keep[8], _I32P), h_final_in=_ptr(h_final))
+        if carried is not None:
+            si.h_prev_in = _ptr(self._keep_c[0])
+            si.prev_len = C.cast(self._keep_c[1], _I32P)
         so = dc_step_out(**{k: _ptr(v) for k, v in self.out.items()})
         if not want_xlogp:
             so.xlogp = None
+        self._keep_h = h_out
+        so.h_out = _ptr(h_out)
         return si, so
 
     def step(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len, remain_len,
-             influence=True, boundary=True, h_final=None, export_kv=False):
+             influence=True, boundary=True, h_final=None, export_kv=False, carried=None,
+             h_out=None):
         """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled.
         export_kv: also append the last block's K / V to the caches (which are then written)."""
         si, so = self._step_structs(k_cache, v_cache, ctx_len, last_ids, last_len, win_ids,
                                     win_len, remain_len, influence, boundary, h_final,
-                                    export_kv=export_kv)
+                                    export_kv=export_kv, carried=carried, h_out=h_out)
         self._check(self._lib.dc_step(self._ctx, C.byref(si), C.byref(so)))
         return self.out
 

@@ -159,6 +159,19 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
   return DC_OK;
 }
 
+// The meta the LM-head stage sees when p_prev is carried in: two variants of LM rows over a stack
+// that ran one.
+SeqMeta carried_meta(const SeqMeta& m, const int32_t* prev_len) {
+  SeqMeta ml = m;
+  ml.nv = 2;
+  const int npos = m.batch * m.W_cap, gmax = 64;
+  ml.G = npos < gmax ? npos : gmax;
+  if (ml.G < 1) ml.G = 1;
+  ml.npos_pad = round_up(npos, ml.G);
+  for (int b = 0; b < m.batch; ++b) ml.have_prev[b] = prev_len[b] > 0 ? 1 : 0;
+  return ml;
+}
+
 #define DC_CHECK_LAUNCH(c)                                                                   \
   do {                                                                                       \
     cudaError_t e_ = cudaGetLastError();                                                     \
@@ -175,7 +188,9 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
   Profiler& pf = c->prof;
   const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
   const int M = m.nv * m.batch * m.R_cap;
-  const int Mlm = m.nv * m.npos_pad;
+  const bool carried = (in->flags & DC_STEP_CARRIED_PREV) != 0;
+  const SeqMeta ml = carried ? carried_meta(m, in->prev_len) : m;   // what the LM-head stage sees
+  const int Mlm = ml.nv * ml.npos_pad;
   const int nqkv = (nq + 2 * nkv) * hd;
   T* a = (T*)c->a; T* q = (T*)c->q; T* k = (T*)c->k; T* v = (T*)c->v; T* o = (T*)c->o;
   T* act = (T*)c->act; T* h = (T*)c->h;
@@ -279,15 +294,21 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     return DC_OK;
   }
   pf.begin(DC_STAGE_NORM, in->h_final_in ? 2 : 1);
-  launch_final_norm<T>(c->x, part, nsplit, part_stride, (const T*)c->final_norm, g.rms_eps, d, m,
-                       h, s);
-  if (in->h_final_in) launch_h_override<T>((const T*)in->h_final_in, g.max_window, d, m, h, s);
+  launch_final_norm<T>(c->x, part, nsplit, part_stride, (const T*)c->final_norm, g.rms_eps, d, ml,
+                       h, s, m.nv);
+  if (carried || out->h_out) {
+    PrevLen pl{};
+    if (carried) for (int b = 0; b < m.batch; ++b) pl.n[b] = in->prev_len[b];
+    launch_carry<T>(carried ? (const T*)in->h_prev_in : nullptr, pl, (T*)out->h_out, g.max_window, d,
+                    ml, h, s);
+  }
+  if (in->h_final_in) launch_h_override<T>((const T*)in->h_final_in, g.max_window, d, ml, h, s);
   pf.end();
 
   SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, g.max_window};
   if (c->tc_lm) {
     pf.begin(DC_STAGE_LMHEAD, 2);
-    int rc = tc_lmhead(c->tc, m, (const __nv_bfloat16*)h, g.mask_id, g.forbid_mask_pred,
+    int rc = tc_lmhead(c->tc, ml, (const __nv_bfloat16*)h, g.mask_id, g.forbid_mask_pred,
                        c->ws_pred, c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so);
     pf.end();
     if (rc != DC_OK) return fail(c, rc, "tensor-core LM head failed: %s", tc_error(c->tc));
@@ -296,26 +317,26 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     pf.begin(DC_STAGE_LMHEAD, 2);
     launch_gemm_simt<T>(h, (const T*)c->lm_head, c->logits, Mlm, g.vocab, d, g.vocab,
                         EPI_STORE_F32, s);
-    launch_signals_from_logits(c->logits, g.vocab, g.mask_id, g.forbid_mask_pred, m, c->ws_pred,
+    launch_signals_from_logits(c->logits, g.vocab, g.mask_id, g.forbid_mask_pred, ml, c->ws_pred,
                                c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so, s);
     pf.end();
     c->have_logits = true;
   }
   if (out->xlogp) {
     pf.begin(DC_STAGE_XLOGP, 1);
-    launch_xlogp<T>(h, (const T*)c->lm_head, c->ws_pred, c->ws_lse, d, m, g.max_window,
+    launch_xlogp<T>(h, (const T*)c->lm_head, c->ws_pred, c->ws_lse, d, ml, g.max_window,
                     out->xlogp, s);
     pf.end();
   }
   if ((in->flags & DC_STEP_BOUNDARY) && out->block_len) {
     pf.begin(DC_STAGE_BOUNDARY, 1);
-    launch_boundary(c->ws_infl, c->ws_ent, m.W_cap, m, c->hp, g.max_window, out->score,
+    launch_boundary(c->ws_infl, c->ws_ent, ml.W_cap, ml, c->hp, g.max_window, out->score,
                     out->cum_influence, out->cum_score, out->block_len, s);
     pf.end();
   }
   if (c->use_tc) tc_flush_status(c->tc, out->status, m.batch);
   DC_CHECK_LAUNCH(c);
-  c->last_meta = m;
+  c->last_meta = ml;
   return DC_OK;
 }
 
@@ -324,8 +345,18 @@ int validate_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, SeqMe
   if (!in || !out) return fail(c, DC_ERR_INVALID_ARG, "null in/out");
   if (!out->status) return fail(c, DC_ERR_INVALID_ARG, "out->status is required");
   if (!in->win_ids || !in->win_len) return fail(c, DC_ERR_INVALID_ARG, "win_ids/win_len null");
-  if (in->flags & ~(DC_STEP_INFLUENCE | DC_STEP_BOUNDARY | DC_STEP_EXPORT_KV))
+  if (in->flags & ~(DC_STEP_INFLUENCE | DC_STEP_BOUNDARY | DC_STEP_EXPORT_KV | DC_STEP_CARRIED_PREV))
     return fail(c, DC_ERR_INVALID_ARG, "unknown flag bits 0x%x", in->flags);
+  if (in->flags & DC_STEP_CARRIED_PREV) {
+    if (in->flags & DC_STEP_INFLUENCE)
+      return fail(c, DC_ERR_INVALID_ARG, "DC_STEP_CARRIED_PREV and DC_STEP_INFLUENCE exclude each other");
+    if (!in->h_prev_in || !in->prev_len)
+      return fail(c, DC_ERR_INVALID_ARG, "DC_STEP_CARRIED_PREV needs h_prev_in and prev_len");
+    for (int b = 0; b < in->batch && b < c->cfg.max_batch; ++b)
+      if (in->prev_len[b] < 0 || in->prev_len[b] > in->win_len[b])
+        return fail(c, DC_ERR_SHAPE, "prev_len[%d]=%d outside [0, win_len=%d]", b, in->prev_len[b],
+                    in->win_len[b]);
+  }
   int rc = build_meta(c, in->batch, in->flags, in->ctx_len, in->last_len, in->win_len,
                       in->remain_len, m);
   if (rc != DC_OK) return rc;

@@ -57,7 +57,13 @@ void launch_rmsnorm(float* x, const float* part, int nsplit, size_t part_stride,
 // final norm of the window rows into the LM-head row order (pad rows are zeroed)
 template <typename T>
 void launch_final_norm(float* x, const float* part, int nsplit, size_t part_stride, const T* g,
-                       float eps, int d, const SeqMeta& m, T* h, cudaStream_t s);
+                       float eps, int d, const SeqMeta& m, T* h, cudaStream_t s, int nv_x = -1);
+// LM rows carried between steps: h_out[b][k] <- curr row (if h_out); prev rows <- h_prev_in[b][k]
+// for k < prev_len.n[b], else the curr row of the same position (if h_prev_in); m.nv must be 2 then
+struct PrevLen { int n[DC_MAX_BATCH]; };
+template <typename T>
+void launch_carry(const T* h_prev_in, const PrevLen& pl, T* h_out, int max_window, int d,
+                  const SeqMeta& m, T* h, cudaStream_t s);
 
 // copy caller-supplied LM-head input [B][2][max_window][d] into the LM-head row order
 template <typename T>

@@ -154,12 +154,13 @@ void launch_rmsnorm(float* x, const float* part, int nsplit, size_t part_stride,
 template <typename T>
 __global__ void k_final_norm(float* __restrict__ x, const float* __restrict__ part, int nsplit,
                              size_t part_stride, const T* __restrict__ g, float eps, int d,
-                             SeqMeta m, T* __restrict__ h) {
+                             SeqMeta m, T* __restrict__ h, int nv_x) {
   __shared__ float red[32];
   // grid: nv * npos_pad LM rows
   const int lrow = blockIdx.x;
   const int grp = lrow / (m.nv * m.G), in = lrow % (m.nv * m.G);
   const int v = in / m.G, p = grp * m.G + in % m.G;
+  if (v >= nv_x) return;   // x holds fewer variants than the LM head sees: those rows are carried in
   T* hr = h + (size_t)lrow * d;
   const int b = p / m.W_cap, k = p % m.W_cap;
   if (b >= m.batch || k >= m.win_len[b]) {
@@ -172,9 +173,51 @@ __global__ void k_final_norm(float* __restrict__ x, const float* __restrict__ pa
 
 template <typename T>
 void launch_final_norm(float* x, const float* part, int nsplit, size_t part_stride, const T* g,
-                       float eps, int d, const SeqMeta& m, T* h, cudaStream_t s) {
-  k_final_norm<T><<<m.nv * m.npos_pad, 256, 0, s>>>(x, part, nsplit, part_stride, g, eps, d, m, h);
+                       float eps, int d, const SeqMeta& m, T* h, cudaStream_t s, int nv_x) {
+  k_final_norm<T><<<m.nv * m.npos_pad, 256, 0, s>>>(x, part, nsplit, part_stride, g, eps, d, m, h,
+                                                    nv_x < 0 ? m.nv : nv_x);
 }
+
+template <typename T>
+__global__ void k_carry(const T* __restrict__ h_prev_in, PrevLen pl, T* __restrict__ h_out,
+                        int max_window, int d, SeqMeta m, T* __restrict__ h) {
+  const int lrow = blockIdx.x;
+  const int grp = lrow / (m.nv * m.G), in = lrow % (m.nv * m.G);
+  const int v = in / m.G, p = grp * m.G + in % m.G;
+  const int b = p / m.W_cap, k = p % m.W_cap;
+  const bool live = b < m.batch && k < m.win_len[b];
+  T* row = h + (size_t)lrow * d;
+  if (v == 0) {
+    if (!live || !h_out) return;
+    T* dst = h_out + ((size_t)b * max_window + k) * d;
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+      float v4[4];
+      load4<T>(row + i, v4);
+      store4<T>(dst + i, v4);
+    }
+    return;
+  }
+  if (!h_prev_in) return;
+  // prev row: the carried row, or (no earlier prediction for this position) the curr row itself,
+  // which makes the two distributions equal and I_k = 0; pad rows are zero
+  const T* src = !live ? nullptr
+               : (k < pl.n[b]) ? h_prev_in + ((size_t)b * max_window + k) * d
+                               : h + (size_t)lm_row(m, 0, p) * d;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float v4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (src) load4<T>(src + i, v4);
+    store4<T>(row + i, v4);
+  }
+}
+
+template <typename T>
+void launch_carry(const T* h_prev_in, const PrevLen& pl, T* h_out, int max_window, int d,
+                  const SeqMeta& m, T* h, cudaStream_t s) {
+  k_carry<T><<<m.nv * m.npos_pad, 128, 0, s>>>(h_prev_in, pl, h_out, max_window, d, m, h);
+}
+template void launch_carry<float>(const float*, const PrevLen&, float*, int, int, const SeqMeta&, float*, cudaStream_t);
+template void launch_carry<__nv_bfloat16>(const __nv_bfloat16*, const PrevLen&, __nv_bfloat16*, int, int,
+                                          const SeqMeta&, __nv_bfloat16*, cudaStream_t);
 
 template <typename T>
 __global__ void k_h_override(const T* __restrict__ h_in, int max_window, int d, SeqMeta m,
@@ -597,7 +640,7 @@ template void launch_export_kv<__nv_bfloat16>(const __nv_bfloat16*, const __nv_b
   template void launch_rmsnorm<T>(float*, const float*, int, size_t, const T*, float, int, int, \
                                   T*, cudaStream_t);                                            \
   template void launch_final_norm<T>(float*, const float*, int, size_t, const T*, float, int,   \
-                                     const SeqMeta&, T*, cudaStream_t);                         \
+                                     const SeqMeta&, T*, cudaStream_t, int);                         \
   template void launch_h_override<T>(const T*, int, int, const SeqMeta&, T*, cudaStream_t);     \
   template void launch_gemm_simt<T>(const T*, const T*, float*, int, int, int, int, int,        \
                                     cudaStream_t);                                              \
