@@ -298,6 +298,9 @@ typedef struct dc_generate_in {
   const int32_t* ctx_len;    /* host [batch]                                                  */
   int32_t gen_len;           /* tokens to decode per sequence, >= 1                           */
   int32_t max_steps;
+  int32_t carried_prev;      /* non-zero: boundary steps take p_prev from the rows the boundary
+                                step before them left (DC_STEP_CARRIED_PREV) instead of running a
+                                second variant                                                */
 } dc_generate_in;
 typedef struct dc_generate_out {
   int32_t* tokens;           /* HOST [batch][gen_len]                                         */

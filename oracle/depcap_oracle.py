@@ -458,7 +458,7 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
 # the decoding loop around the step (Section 3, Eq. 1-2; Section 4.2; Algorithm 1 per step)
 # ------------------------------------------------------------------------------------------
 def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, gen_len: int,
-             max_window: int, max_steps: int | None = None) -> dict:
+             max_window: int, max_steps: int | None = None, carried: bool = False) -> dict:
     """Decode gen_len tokens after a cached context, one sequence.
 
     Every stage (Section 4.2): from the frontier, one forward over the last decoded block
@@ -468,6 +468,8 @@ def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, ge
     same forward's predictions already serve the new block: Algorithm 1 picks the subset of
     [0, L) to commit (Eq. 2).  Then the block's L positions are denoised alone - forward,
     Algorithm 1, Eq. 2 - until no [MASK] is left; the block becomes the last decoded block.
+    carried: the boundary step takes p_prev from the LM-head rows the boundary step before it
+    left for the same positions (rows L.. of its window) instead of a second pass.
     Returns tokens [gen_len], block_lens (list), nfe (forwards of the curr variant = steps) and
     a per-step trace (kind, pred, conf, selected, block_len, score, ids after the commit).
     """
@@ -485,6 +487,7 @@ def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, ge
     block_lens: list[int] = []
     trace: list[dict] = []
     nfe = 0
+    carry_rows = np.zeros((0, cfg.d_model))
     limit = 4 * gen_len if not max_steps or max_steps <= 0 else max_steps
     while len(tokens) < gen_len:
         remaining = gen_len - len(tokens)
@@ -493,7 +496,11 @@ def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, ge
             raise RuntimeError("max_steps reached")
         W = min(cfg.L_max, max_window, remaining)
         win = np.full(W, cfg.mask_id, dtype=np.int64)
-        r = step(cfg, w, kc, vc, cache, last, win, remaining, influence=True, return_kv=True)
+        if carried:
+            r = step(cfg, w, kc, vc, cache, last, win, remaining, return_kv=True,
+                     carried=(carry_rows, min(len(carry_rows), W)))
+        else:
+            r = step(cfg, w, kc, vc, cache, last, win, remaining, influence=True, return_kv=True)
         nfe += 1
         for l in range(n_l):        # the last block moves into the cache
             k_l, v_l = r["kv_last"][l]
@@ -503,6 +510,7 @@ def generate(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int, ge
         cache += len(last)
         last = np.zeros(0, dtype=np.int64)
         L = int(r["block_len"])
+        carry_rows = r["h_curr"][L:]
         block_lens.append(L)
         for i in r["selected"]:
             win[i] = r["pred"][i]

@@ -107,7 +107,8 @@ class dc_commit_out(C.Structure):
 
 class dc_generate_in(C.Structure):
     _fields_ = [("batch", C.c_int32), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
-                ("ctx_len", _I32P), ("gen_len", C.c_int32), ("max_steps", C.c_int32)]
+                ("ctx_len", _I32P), ("gen_len", C.c_int32), ("max_steps", C.c_int32),
+                ("carried_prev", C.c_int32)]
 
 
 class dc_generate_out(C.Structure):
@@ -415,7 +416,7 @@ class DepCap:
         self._check(self._lib.dc_commit(self._ctx, C.byref(ci), C.byref(co)))
         return self._remaining
 
-    def generate(self, k_cache, v_cache, ctx_len, gen_len, max_steps=0):
+    def generate(self, k_cache, v_cache, ctx_len, gen_len, max_steps=0, carried_prev=False):
         """Block-wise generation (host arrays out): tokens [B, gen_len], block_lens, nfe."""
         B = len(ctx_len)
         cl_ = _host_i32(ctx_len, B)
@@ -423,7 +424,8 @@ class DepCap:
         blocks = (C.c_int32 * (B * gen_len))()
         nfe = (C.c_int32 * 1)()
         gi = dc_generate_in(batch=B, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
-                            ctx_len=C.cast(cl_, _I32P), gen_len=gen_len, max_steps=max_steps)
+                            ctx_len=C.cast(cl_, _I32P), gen_len=gen_len, max_steps=max_steps,
+                            carried_prev=int(carried_prev))
         go = dc_generate_out(tokens=C.cast(tokens, _I32P), block_lens=C.cast(blocks, _I32P),
                              nfe=C.cast(nfe, _I32P))
         self._check(self._lib.dc_generate(self._ctx, C.byref(gi), C.byref(go)))

@@ -89,6 +89,7 @@ struct dc_ctx {
   int32_t *g_win = nullptr, *g_last = nullptr, *g_pred = nullptr, *g_blk = nullptr, *g_cnt = nullptr,
           *g_idx = nullptr, *g_rem = nullptr, *g_status = nullptr;
   float *g_conf = nullptr, *g_xlogp = nullptr;
+  char *g_hout = nullptr, *g_carry = nullptr;   // LM-head rows of a boundary step / kept for the next one
   uint8_t* g_mask = nullptr;
   SeqMeta last_meta{};
   bool have_logits = false;
@@ -503,6 +504,9 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
     c->g_cnt = ws_alloc<int32_t>(c, g.max_batch, &ok);
     c->g_rem = ws_alloc<int32_t>(c, g.max_batch, &ok);
     c->g_status = ws_alloc<int32_t>(c, g.max_batch, &ok);
+    const size_t hbytes = nw * g.d_model * (g.dtype == DC_BF16 ? 2 : 4);
+    c->g_hout = ws_alloc<char>(c, hbytes, &ok);
+    c->g_carry = ws_alloc<char>(c, hbytes, &ok);
   }
   if (c->use_tc) {
     int rc = tc_create(g, c->stream, c->M_max, c->Mlm_max, c->wq, c->wk, c->wv, c->wo, c->w_gate,
@@ -634,11 +638,14 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
   if ((!in->k_cache || !in->v_cache)) return fail(c, DC_ERR_INVALID_ARG, "k_cache / v_cache null");
   const int max_steps = in->max_steps > 0 ? in->max_steps : 4 * N;
 
-  struct Seq { int cache, done, blk, last_len, nblocks; };   // cache: keys in the cache; done: tokens decoded
+  struct Seq { int cache, done, blk, last_len, nblocks, carry; };   // cache: keys in the cache; done: tokens decoded; carry: rows kept for p_prev
+  const bool carried = in->carried_prev != 0;
+  const size_t row_bytes = (size_t)g.d_model * (c->bf16 ? 2 : 4);
+  std::vector<int32_t> h_prevlen(B);
   std::vector<Seq> sq(B);
   std::vector<int32_t> h_ctx(B), h_lastlen(B), h_winlen(B), h_remain(B), h_blk(B), h_rem(B);
   std::vector<int32_t> h_win((size_t)B * MW), h_last((size_t)B * (g.max_last > 0 ? g.max_last : 1));
-  for (int b = 0; b < B; ++b) sq[b] = Seq{in->ctx_len[b], 0, 0, 0, 0};
+  for (int b = 0; b < B; ++b) sq[b] = Seq{in->ctx_len[b], 0, 0, 0, 0, 0};
   if (out->block_lens) memset(out->block_lens, 0, sizeof(int32_t) * (size_t)B * N);
   cudaStream_t s = c->stream;
   int nfe = 0;
@@ -660,6 +667,7 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
       } else if (q.blk == 0) {                 // boundary step: all of the look-ahead window masked
         const int W = (N - q.done) < Lw_cap ? (N - q.done) : Lw_cap;
         h_lastlen[b] = q.last_len; h_winlen[b] = W;
+        h_prevlen[b] = q.carry < W ? q.carry : W;
         for (int i = 0; i < W; ++i) h_win[(size_t)b * MW + i] = g.mask_id;
       } else {                                 // denoising step inside the block: ids live on the device
         h_lastlen[b] = 0; h_winlen[b] = q.blk;
@@ -673,13 +681,20 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
       cudaMemcpyAsync(c->g_last, h_last.data(), sizeof(int32_t) * h_last.size(), cudaMemcpyHostToDevice, s);
     dc_step_in si{};
     si.batch = B;
-    si.flags = any_boundary ? (DC_STEP_INFLUENCE | DC_STEP_BOUNDARY | DC_STEP_EXPORT_KV) : 0;
+    si.flags = any_boundary ? ((carried ? DC_STEP_CARRIED_PREV : DC_STEP_INFLUENCE) | DC_STEP_BOUNDARY |
+                               DC_STEP_EXPORT_KV) : 0;
+    if (any_boundary && carried) {
+      for (int b = 0; b < B; ++b)
+        if (!(sq[b].done < N && sq[b].blk == 0)) h_prevlen[b] = 0;
+      si.h_prev_in = c->g_carry; si.prev_len = h_prevlen.data();
+    }
     si.k_cache = in->k_cache; si.v_cache = in->v_cache; si.ctx_len = h_ctx.data();
     si.last_ids = c->g_last; si.last_len = h_lastlen.data();
     si.win_ids = c->g_win; si.win_len = h_winlen.data(); si.remain_len = h_remain.data();
     dc_step_out so{};
     so.pred_id = c->g_pred; so.conf = c->g_conf; so.xlogp = c->g_xlogp; so.status = c->g_status;
     so.block_len = any_boundary ? c->g_blk : nullptr;
+    so.h_out = (any_boundary && carried) ? c->g_hout : nullptr;
     int rc = dc_step(c, &si, &so);
     if (rc != DC_OK) return rc;
     ++nfe;
@@ -717,6 +732,13 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
         q.blk = h_blk[b];
         if (out->block_lens) out->block_lens[(size_t)b * N + q.nblocks] = q.blk;
         ++q.nblocks;
+        if (carried) {   // rows blk .. W of this window are rows 0 .. of the next one
+          q.carry = h_winlen[b] - q.blk;
+          if (q.carry > 0)
+            cudaMemcpyAsync(c->g_carry + (size_t)b * MW * row_bytes,
+                            c->g_hout + ((size_t)b * MW + q.blk) * row_bytes, (size_t)q.carry * row_bytes,
+                            cudaMemcpyDeviceToDevice, s);
+        }
       }
       if (h_rem[b] == 0) {                     // block complete: read its ids back
         if (cudaMemcpyAsync(out->tokens + (size_t)b * N + q.done, c->g_win + (size_t)b * MW,

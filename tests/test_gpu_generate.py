@@ -113,6 +113,25 @@ def test_generation_fp32_matches_the_oracle(lam, norm):
     eng.close()
 
 
+@pytest.mark.parametrize("lam,norm", [(0.02, 2), (0.3, 1)])
+def test_generation_with_carried_prev_matches_the_oracle(lam, norm):
+    """The same generations with p_prev carried from boundary step to boundary step (one variant
+    through the stack): identical tokens, block lengths and forward count."""
+    hy = Hyper(tau_low=0.3, tau_high=0.6, lam=lam, norm_mode=norm, L_min=4, L_max=16)
+    case = _peaked(TINY, hy)
+    N = 48
+    ref = O.generate(case.ocfg, case.ow, adapters.to_np(case.k_log[:, 0]),
+                     adapters.to_np(case.v_log[:, 0]), 64, N, 32, carried=True)
+    assert len(set(ref["block_lens"])) > 1
+    eng = case.make_engine(max_ctx=128, max_last=16, max_window=32)
+    di = case.device_inputs(eng)
+    tok, blocks, nfe = eng.generate(di["k_cache"], di["v_cache"], [64], N, carried_prev=True)
+    assert blocks[0] == ref["block_lens"]
+    assert tok[0].tolist() == ref["tokens"].tolist()
+    assert nfe == ref["nfe"]
+    eng.close()
+
+
 def test_generation_batch_of_independent_sequences():
     """Two sequences with different contexts advance independently: each equals its own
     single-sequence oracle run; NFE is the longer of the two."""

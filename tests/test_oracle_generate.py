@@ -113,3 +113,21 @@ def test_against_a_brute_force_sequential_decoder():
         out.extend(blk.tolist())
         last = blk.copy()
     assert out == r["tokens"].tolist()
+
+
+def test_carried_prev_generation_keeps_the_structure_and_the_cold_start():
+    """With p_prev carried between boundary steps the loop has the same structure; the first block
+    is the cold start, and a later block never reaches beyond the positions that had a carried
+    row (window of the boundary step before it, minus its block)."""
+    hy = Hyper(tau_low=0.3, tau_high=0.6, lam=0.8, norm_mode=2, L_min=4, L_max=16)
+    case, kc, vc = _case(hy)
+    r = O.generate(case.ocfg, case.ow, kc, vc, 64, 48, 32, carried=True)
+    assert sum(r["block_lens"]) == 48 and not np.any(r["tokens"] == TINY.mask_id)
+    assert r["block_lens"][0] == hy.L_min
+    done, prev_w = 0, None
+    for i, L in enumerate(r["block_lens"]):
+        W = min(hy.L_max, 48 - done, 32)
+        if i > 0:
+            carried_rows = prev_w - r["block_lens"][i - 1]
+            assert L <= max(min(carried_rows, W), min(hy.L_min, W))
+        prev_w, done = W, done + L
