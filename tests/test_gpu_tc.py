@@ -92,3 +92,37 @@ def test_fused_dense_chain_is_the_path_taken_when_the_rows_fit_one_block():
         else:
             assert launches["dense"] == 0 and launches["qkv"] == case.n_layers
         eng.close()
+
+
+@pytest.mark.parametrize("last,win,influence,rows", [(32, 96, True, 256), (0, 16, True, 32), (0, 32, False, 32)])
+def test_fused_chain_at_its_row_limits(last, win, influence, rows):
+    """The fused chain takes 32 .. 256 activation rows: both ends, against the oracle."""
+    wl = _wl(1, last=max(last, 1), win=win)
+    lengths = dict(ctx_len=[100], last_len=[last], win_len=[win], remain_len=[128])
+    case = Case(wl, lengths=lengths)
+    eng = case.make_engine(max_window=(win + 15) // 16 * 16)
+    di = case.device_inputs(eng)
+    out = eng.step(influence=influence, boundary=True, **di)
+    sel = eng.select(di["win_ids"], di["win_len"])
+    eng.synchronize()
+    gpu = {k_: v_.cpu().numpy() for k_, v_ in out.items()}
+    gpu.update({k_: v_.cpu().numpy() for k_, v_ in sel.items()})
+    compare(case, gpu, case.run_oracle(influence=influence))
+    _, launches = eng.step_profiled(influence=influence, boundary=True, **di)
+    assert launches["dense"] == case.n_layers + 1, rows
+    eng.close()
+
+
+@pytest.mark.parametrize("n_q,n_kv", [(40, 20), (28, 4), (6, 2)])
+def test_fused_chain_qkv_helper_layouts(n_q, n_kv):
+    """The balanced QKV phase with 80 tiles (34 helper pairs, six of which serve two tile pairs),
+    36 tiles (Dream's head counts: one tile pair per helper, helpers left over) and 10 tiles."""
+    wl = _wl(1, n_q=n_q, n_kv=n_kv, d=512, ff=1024, vocab=2048, layers=2)
+    case = Case(wl)
+    eng = case.make_engine()
+    gpu, ora = case.run_gpu(eng), case.run_oracle()
+    compare(case, gpu, ora)
+    di = case.device_inputs(eng)
+    _, launches = eng.step_profiled(**di)
+    assert launches["dense"] == case.n_layers + 1
+    eng.close()
