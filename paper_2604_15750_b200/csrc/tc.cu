@@ -454,8 +454,9 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
       cudaStreamSynchronize(t->s);
       cudaMemcpy(trace_buf, trace_dev, 256 * 64 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
       ++n_print;
-      char fn[64];
-      snprintf(fn, sizeof(fn), "gpurun_out/chain_trace_dbg%s_%d.txt", getenv("DC_TAG") ? getenv("DC_TAG") : "0", n_print);
+      char fn[256];
+      snprintf(fn, sizeof(fn), "%s/chain_trace_dbg%s_%d.txt", getenv("DC_TRACE_DIR") ? getenv("DC_TRACE_DIR") : ".",
+               getenv("DC_TAG") ? getenv("DC_TAG") : "0", n_print);
       FILE* f = fopen(fn, "w");
       if (f) {
         for (int c = 0; c < t->chain_grid; ++c) {
