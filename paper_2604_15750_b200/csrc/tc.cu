@@ -299,7 +299,14 @@ static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
   if (stages > 8) stages = 8;
   if (stages < 2) return tfail(t, DC_ERR_UNSUPPORTED, "activation block too large for the smem ring");
   const size_t smem = (size_t)stages * sb + 1024;
-  dim3 grid(tiles * ((p.M + p.BN - 1) / p.BN), p.nsplit, 1);
+  // persistent: one CTA per SM works through the units; with more units than CTAs the
+  // accumulators of consecutive units alternate between two TMEM sets
+  const int n_units = tiles * ((p.M + p.BN - 1) / p.BN) * p.nsplit;
+  const int grid = n_units < t->n_sm ? n_units : t->n_sm;
+  p.tiles = tiles;
+  // gate / up keep both TMEM sets for one unit (column blocks of 256 rows: with 128-row blocks
+  // every weight tile is pulled from L2 twice as often, which cost more than the overlap gained)
+  p.pingpong = (n_units > grid && nw == 1) ? 1 : 0;
   p.status = t->status;
   k_gemm_tc<EPI><<<grid, kGemmThreads, smem, t->s>>>(w0, w1, w2, ma, p, stages);
   cudaError_t e = cudaGetLastError();

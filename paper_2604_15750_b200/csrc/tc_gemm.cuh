@@ -12,6 +12,16 @@
 // warps 2..5 = epilogue (TMEM -> registers -> global).  Shared memory is a ring of kStages
 // slots, each {NW weight tiles 128 x 64, one activation tile BN x 64}, all in the 128-byte
 // swizzled K-major layout that both TMA and tcgen05.mma understand.
+//
+// A CTA works through the units (weight tile, column block, K split) blockIdx.x, + gridDim.x, ...
+// With more units than CTAs (`pingpong`) the accumulators of consecutive units alternate
+// between two TMEM sets, the producer and the MMA issuer run on into the next unit, and the
+// epilogue of a unit - which took 25..60% of a unit's time when every unit was a CTA of its own -
+// runs under the MMAs of the next.  A set is one accumulator of up to 256 columns (at N = 256 a
+// single chain of MMAs already runs at the tensor core's rate).  Without `pingpong` (one unit per
+// CTA, or gate / up, which need both sets for one unit) both sets serve a unit - even / odd
+// k-steps, because small N needs two independent chains, or gate / up - and a CTA's next unit
+// starts when the epilogue has drained them.
 #pragma once
 #include "kernels.h"
 #include "tc_ptx.cuh"
@@ -30,6 +40,8 @@ struct GemmParams {
   int K;          // reduction length
   int BN;         // activation rows per column block (multiple of 16, <= 256)
   int nsplit;     // split-K factor
+  int tiles;      // weight tiles (over all matrices of the call)
+  int pingpong;   // more units than CTAs: one accumulator set per unit, sets alternate
   // QKV epilogue
   int nq, nkv, hd;          // tiles [0,nq) are q heads, [nq,nq+nkv) k heads, rest v heads
   const float* cos_sin;     // RoPE table [(b, r)][hd]
@@ -59,7 +71,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           const GemmParams p, const int stages) {
   constexpr int NW = (EPI == GEMM_EPI_SWIGLU) ? 2 : 1;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bar_full[8], bar_empty[8], bar_acc;
+  __shared__ uint64_t bar_full[8], bar_empty[8], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float xch[(EPI == GEMM_EPI_QKV) ? 128 * 33 : 1];
@@ -67,35 +79,45 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Column blocks of one weight tile sit next to each other in the launch order, so that the
+  // Column blocks of one weight tile sit next to each other in the unit order, so that the
   // CTAs that share a weight tile run together and all but one read it from L2.
   const int n_cblk = (p.M + p.BN - 1) / p.BN;
-  const int tile = blockIdx.x / n_cblk;   // weight tile
-  const int cblk = blockIdx.x % n_cblk;   // activation column block
-  const int split = blockIdx.y;           // K split
+  const int per_split = p.tiles * n_cblk;
+  const int n_units = per_split * p.nsplit;
   const int stage_bytes = gemm_stage_bytes(NW, p.BN);
   const int KB = p.K / kTileK;
-  const int kb0 = (int)(((long long)split * KB) / p.nsplit);
-  const int kb1 = (int)(((long long)(split + 1) * KB) / p.nsplit);
-  const int nkb = kb1 - kb0;
-  const uint32_t tmem_cols = 512u;   // two accumulators of up to 256 columns
+  const bool pp = p.pingpong != 0;
+  const uint32_t up_off = pp ? 128u : 256u;   // second accumulator of a set (gate / up), or the odd k-steps' one
+  const uint32_t tmem_cols = 512u;
 
-  // which weight matrix and which row of it this tile starts at
-  const CUtensorMap* map_w = &map_w0;
-  int wrow = tile * kTileN;
-  if (EPI == GEMM_EPI_QKV) {
-    if (tile >= p.nq + p.nkv) { map_w = &map_w2; wrow = (tile - p.nq - p.nkv) * kTileN; }
-    else if (tile >= p.nq) { map_w = &map_w1; wrow = (tile - p.nq) * kTileN; }
-  }
+  struct Unit { int tile, cblk, split, kb0, nkb, wrow; const CUtensorMap* map_w; };
+  auto unit_of = [&](int u) {
+    Unit w;
+    w.split = u / per_split;
+    const int rem = u - w.split * per_split;
+    w.tile = rem / n_cblk;
+    w.cblk = rem - w.tile * n_cblk;
+    w.kb0 = (int)(((long long)w.split * KB) / p.nsplit);
+    w.nkb = (int)(((long long)(w.split + 1) * KB) / p.nsplit) - w.kb0;
+    // which weight matrix and which row of it this tile starts at
+    w.map_w = &map_w0;
+    w.wrow = w.tile * kTileN;
+    if (EPI == GEMM_EPI_QKV) {
+      if (w.tile >= p.nq + p.nkv) { w.map_w = &map_w2; w.wrow = (w.tile - p.nq - p.nkv) * kTileN; }
+      else if (w.tile >= p.nq) { w.map_w = &map_w1; w.wrow = (w.tile - p.nq) * kTileN; }
+    }
+    return w;
+  };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int i = 0; i < stages; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
-    ptx::mbar_init(&bar_acc, 1);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128); }
     ptx::fence_barrier_init();
-    ptx::prefetch_tmap(map_w);
+    ptx::prefetch_tmap(&map_w0);
     ptx::prefetch_tmap(&map_a);
-    if (NW == 2) ptx::prefetch_tmap(&map_w1);
+    if (NW == 2 || EPI == GEMM_EPI_QKV) ptx::prefetch_tmap(&map_w1);
+    if (EPI == GEMM_EPI_QKV) ptx::prefetch_tmap(&map_w2);
   }
   if (warp == 1) {
     ptx::tmem_alloc(&tmem_base_s, tmem_cols);
@@ -113,63 +135,91 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     if (lane == 0) {
       const uint32_t ring0 = ptx::smem_u32(smem);
       const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
-      const int arow = cblk * p.BN;
       uint32_t s = 0, ph = 0, slot = ring0;
-      for (int i = 0; i < nkb; ++i) {
-        if (!ptx::mbar_wait_a(empty0 + 8u * s, ph ^ 1u, &abort_flag)) break;
-        ptx::mbar_expect_tx_a(full0 + 8u * s, (uint32_t)stage_bytes);
-        const int kc = (kb0 + i) * kTileK;
-        ptx::tma_load_2d_a(slot, map_w, full0 + 8u * s, kc, wrow);
-        if (NW == 2) ptx::tma_load_2d_a(slot + kTileN * kTileK * 2, &map_w1, full0 + 8u * s, kc, wrow);
-        ptx::tma_load_2d_a(slot + NW * kTileN * kTileK * 2, &map_a, full0 + 8u * s, kc, arow);
-        if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const Unit w = unit_of(u);
+        const int arow = w.cblk * p.BN;
+        for (int i = 0; i < w.nkb; ++i) {
+          if (!ptx::mbar_wait_a(empty0 + 8u * s, ph ^ 1u, &abort_flag)) { ok = false; break; }
+          ptx::mbar_expect_tx_a(full0 + 8u * s, (uint32_t)stage_bytes);
+          const int kc = (w.kb0 + i) * kTileK;
+          ptx::tma_load_2d_a(slot, w.map_w, full0 + 8u * s, kc, w.wrow);
+          if (NW == 2) ptx::tma_load_2d_a(slot + kTileN * kTileK * 2, &map_w1, full0 + 8u * s, kc, w.wrow);
+          ptx::tma_load_2d_a(slot + NW * kTileN * kTileK * 2, &map_a, full0 + 8u * s, kc, arow);
+          if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
+        }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    // Two accumulators (TMEM columns 0.. and 256..) alternate so that consecutive MMAs do not
-    // depend on each other: gate / up have one each, the other epilogues get even k-steps in
-    // the first and odd k-steps in the second and add them.
     if (lane == 0) {
       const uint32_t idesc = ptx::idesc_bf16(kTileN, p.BN);
       const uint32_t ring0 = ptx::smem_u32(smem);
       const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
       const uint64_t hi = ptx::smem_desc_sw128_hi();
-      uint32_t s = 0, ph = 0, slot = ring0, acc_first = 0;
-      for (int i = 0; i < nkb; ++i) {
-        if (!ptx::mbar_wait_a(full0 + 8u * s, ph, &abort_flag)) break;
-        const uint64_t dw0 = hi | (uint64_t)(slot >> 4);
-        const uint64_t dw1 = dw0 + (kTileN * kTileK * 2 >> 4);
-        const uint64_t da = dw0 + (NW * kTileN * kTileK * 2 >> 4);
-        if (NW == 2) {
-          ptx::umma_bf16(tmem_base, dw0, da, idesc, acc_first);
-          ptx::umma_bf16(tmem_base + 256, dw1, da, idesc, acc_first);
-#pragma unroll
-          for (int kk = 1; kk < kTileK / 16; ++kk) {
-            ptx::umma_bf16_acc(tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
-            ptx::umma_bf16_acc(tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
-          }
-        } else {
-          ptx::umma_bf16(tmem_base, dw0, da, idesc, acc_first);
-          ptx::umma_bf16(tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
-          ptx::umma_bf16_acc(tmem_base, dw0 + 4, da + 4, idesc);
-          ptx::umma_bf16_acc(tmem_base + 256, dw0 + 6, da + 6, idesc);
+      uint32_t s = 0, ph = 0, slot = ring0;
+      bool ok = true;
+      int j = 0;   // units of this CTA so far
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++j) {
+        const Unit w = unit_of(u);
+        const uint32_t set = pp ? (uint32_t)(j & 1) : 0u;
+        // the epilogue has drained this set (its use before the last one)
+        if (j >= (pp ? 2 : 1)) {
+          const uint32_t uses = pp ? (uint32_t)(j >> 1) : (uint32_t)j;   // completed uses of the set
+          if (!ptx::mbar_wait(&acc_empty[set], (uses - 1) & 1u, &abort_flag)) { ok = false; break; }
         }
-        acc_first = 1;
-        ptx::umma_commit_a(empty0 + 8u * s);  // slot free once these MMAs have read it
-        if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
+        ptx::tc_fence_after();
+        const uint32_t acc0 = tmem_base + set * 256u, acc1 = acc0 + up_off;
+        uint32_t acc_first = 0;
+        for (int i = 0; i < w.nkb; ++i) {
+          if (!ptx::mbar_wait_a(full0 + 8u * s, ph, &abort_flag)) { ok = false; break; }
+          const uint64_t dw0 = hi | (uint64_t)(slot >> 4);
+          const uint64_t dw1 = dw0 + (kTileN * kTileK * 2 >> 4);
+          const uint64_t da = dw0 + (NW * kTileN * kTileK * 2 >> 4);
+          if (NW == 2) {
+            ptx::umma_bf16(acc0, dw0, da, idesc, acc_first);
+            ptx::umma_bf16(acc1, dw1, da, idesc, acc_first);
+#pragma unroll
+            for (int kk = 1; kk < kTileK / 16; ++kk) {
+              ptx::umma_bf16_acc(acc0, dw0 + 2 * kk, da + 2 * kk, idesc);
+              ptx::umma_bf16_acc(acc1, dw1 + 2 * kk, da + 2 * kk, idesc);
+            }
+          } else if (pp) {
+            ptx::umma_bf16(acc0, dw0, da, idesc, acc_first);
+            ptx::umma_bf16_acc(acc0, dw0 + 2, da + 2, idesc);
+            ptx::umma_bf16_acc(acc0, dw0 + 4, da + 4, idesc);
+            ptx::umma_bf16_acc(acc0, dw0 + 6, da + 6, idesc);
+          } else {
+            ptx::umma_bf16(acc0, dw0, da, idesc, acc_first);
+            ptx::umma_bf16(acc1, dw0 + 2, da + 2, idesc, acc_first);
+            ptx::umma_bf16_acc(acc0, dw0 + 4, da + 4, idesc);
+            ptx::umma_bf16_acc(acc1, dw0 + 6, da + 6, idesc);
+          }
+          acc_first = 1;
+          ptx::umma_commit_a(empty0 + 8u * s);  // slot free once these MMAs have read it
+          if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
+        }
+        if (ok) ptx::umma_commit(&acc_full[set]);   // this unit's accumulators are complete
       }
-      ptx::umma_commit(&bar_acc);         // accumulators complete
     }
   } else {
     // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
     const int quarter = warp & 3;
     const int f = quarter * 32 + lane;  // feature (weight row) inside the tile = TMEM lane
-    const bool ok = ptx::mbar_wait(&bar_acc, 0, &abort_flag);
-    ptx::tc_fence_after();
-    if (ok && nkb > 0) {
-      const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      const int m_base = cblk * p.BN;
+    bool ok = true;
+    int j = 0;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++j) {
+      const Unit w = unit_of(u);
+      const int tile = w.tile, split = w.split;
+      const uint32_t set = pp ? (uint32_t)(j & 1) : 0u;
+      const uint32_t uses = pp ? (uint32_t)(j >> 1) : (uint32_t)j;
+      ok = ptx::mbar_wait(&acc_full[set], uses & 1u, &abort_flag);
+      ptx::tc_fence_after();
+      if (!ok) break;
+      if (w.nkb > 0) {
+      const uint32_t t_lane = tmem_base + set * 256u + ((uint32_t)(quarter * 32) << 16);
+      const int m_base = w.cblk * p.BN;
       for (int c0 = 0; c0 < p.BN; c0 += 32) {
         float acc[32];
         // BN is a multiple of 16: the last chunk may be 16 wide
@@ -179,22 +229,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           float a16[16];
           ptx::tmem_ld_32x16(t_lane + c0, a16);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) { acc[j] = a16[j]; acc[16 + j] = 0.f; }
+          for (int j2 = 0; j2 < 16; ++j2) { acc[j2] = a16[j2]; acc[16 + j2] = 0.f; }
         }
         ptx::tmem_ld_wait();
-        if (EPI != GEMM_EPI_SWIGLU) {
+        if (EPI != GEMM_EPI_SWIGLU && !pp) {
           // odd k-steps went to the second accumulator
           float odd[32];
-          if (width == 32) ptx::tmem_ld_32x32(t_lane + 256 + c0, odd);
+          if (width == 32) ptx::tmem_ld_32x32(t_lane + up_off + c0, odd);
           else {
             float a16[16];
-            ptx::tmem_ld_32x16(t_lane + 256 + c0, a16);
+            ptx::tmem_ld_32x16(t_lane + up_off + c0, a16);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) { odd[j] = a16[j]; odd[16 + j] = 0.f; }
+            for (int j2 = 0; j2 < 16; ++j2) { odd[j2] = a16[j2]; odd[16 + j2] = 0.f; }
           }
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] += odd[j];
+          for (int j2 = 0; j2 < 32; ++j2) acc[j2] += odd[j2];
         }
         if (EPI == GEMM_EPI_PARTIAL) {
           float* dst = p.part + (size_t)split * p.part_stride + (size_t)(tile * kTileN + f);
@@ -205,10 +255,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           }
         } else if (EPI == GEMM_EPI_SWIGLU) {
           float up[32];
-          if (width == 32) ptx::tmem_ld_32x32(t_lane + 256 + c0, up);
+          if (width == 32) ptx::tmem_ld_32x32(t_lane + up_off + c0, up);
           else {
             float a16[16];
-            ptx::tmem_ld_32x16(t_lane + 256 + c0, a16);
+            ptx::tmem_ld_32x16(t_lane + up_off + c0, a16);
 #pragma unroll
             for (int j = 0; j < 16; ++j) { up[j] = a16[j]; up[16 + j] = 0.f; }
           }
@@ -277,6 +327,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           }
         }
       }
+      }
+      // the set may be overwritten by the unit after the next
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&acc_empty[set]);
     }
   }
   ptx::tc_fence_before();
