@@ -102,6 +102,7 @@ struct TcState {
   unsigned int* grid_bar = nullptr;  // arrival counter of the dense chain's grid barrier, then kFlagWords tile flags
   unsigned int qkv_launches = 0;     // chain launches of this step that ran a QKV phase
   bool balance_qkv = true;
+  bool gemm_pairs = true;            // per-op GEMMs on CTA pairs when there are several column blocks
   unsigned int bar_count = 0;        // arrivals the launches of this step have used up so far
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
   bool chain_coop = false;           // launched cooperatively (co-residency guaranteed)
@@ -221,15 +222,24 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
     cudaGetLastError();
     return tfail(t, DC_ERR_CUDA, "cannot opt in to %d bytes of shared memory", kAttnSmem);
   }
-  cudaError_t e1 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_QKV>,
+  cudaError_t e1 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_QKV, false>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kSmemBudget + 1024 - kStaticQkv);
-  cudaError_t e2 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_PARTIAL>,
+  cudaError_t e2 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_PARTIAL, false>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kSmemBudget + 1024 - kStaticOther);
-  cudaError_t e3 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_SWIGLU>,
+  cudaError_t e3 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_SWIGLU, false>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kSmemBudget + 1024 - kStaticOther);
+  if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_QKV, true>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   kSmemBudget + 1024 - kStaticQkv);
+  if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_PARTIAL, true>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   kSmemBudget + 1024 - kStaticOther);
+  if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(k_gemm_tc<GEMM_EPI_SWIGLU, true>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   kSmemBudget + 1024 - kStaticOther);
   if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
     cudaGetLastError();
     return tfail(t, DC_ERR_CUDA, "cannot opt in to %d bytes of shared memory", kSmemBudget);
@@ -264,6 +274,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
         if (e_ && e_[0] == '0') t->chain_coop = false;
         e_ = getenv("DC_BALANCE_QKV");   // DC_BALANCE_QKV=0: every QKV tile by its owner alone
         if (e_ && e_[0] == '0') t->balance_qkv = false;
+        e_ = getenv("DC_GEMM_PAIRS");    // DC_GEMM_PAIRS=0: per-op GEMMs on single CTAs
+        if (e_ && e_[0] == '0') t->gemm_pairs = false;
       }
     }
     cudaGetLastError();
@@ -289,28 +301,50 @@ static int get_act_maps(TcState* t, const __nv_bfloat16* a, int BN, ActMaps** ou
   return DC_OK;
 }
 
+// ma: activation map with a box of BN rows; ma_half: with BN / 2 rows (CTA pairs), or null
 template <int EPI>
 static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
-                       const CUtensorMap& w2, const CUtensorMap& ma, GemmParams p, int tiles,
-                       int static_smem) {
+                       const CUtensorMap& w2, const CUtensorMap& ma, const CUtensorMap* ma_half,
+                       GemmParams p, int tiles, int static_smem) {
   const int nw = (EPI == GEMM_EPI_SWIGLU) ? 2 : 1;
-  const int sb = gemm_stage_bytes(nw, p.BN);
+  const int n_cblk = (p.M + p.BN - 1) / p.BN;
+  // CTA pairs (each CTA stages half of the activation block) when the shapes allow it and there
+  // is more than one column block: below that the fused chain is the path that matters
+  const bool pair = t->gemm_pairs && ma_half != nullptr && tiles % 2 == 0 && p.BN % 32 == 0 &&
+                    p.BN >= 64 && n_cblk > 1 && t->n_sm >= 2;
+  const int sb = gemm_stage_bytes(nw, pair ? p.BN / 2 : p.BN);
   int stages = (kSmemBudget - static_smem) / sb;
   if (stages > 8) stages = 8;
   if (stages < 2) return tfail(t, DC_ERR_UNSUPPORTED, "activation block too large for the smem ring");
   const size_t smem = (size_t)stages * sb + 1024;
-  // persistent: one CTA per SM works through the units; with more units than CTAs the
-  // accumulators of consecutive units alternate between two TMEM sets
-  const int n_units = tiles * ((p.M + p.BN - 1) / p.BN) * p.nsplit;
-  const int grid = n_units < t->n_sm ? n_units : t->n_sm;
+  // persistent: one CTA (pair) per SM (pair) works through the units; with more units than
+  // workers the accumulators of consecutive units alternate between two TMEM sets
+  const int n_units = (pair ? tiles / 2 : tiles) * n_cblk * p.nsplit;
+  const int workers_max = pair ? t->n_sm / 2 : t->n_sm;
+  const int workers = n_units < workers_max ? n_units : workers_max;
   p.tiles = tiles;
   // gate / up keep both TMEM sets for one unit (column blocks of 256 rows: with 128-row blocks
   // every weight tile is pulled from L2 twice as often, which cost more than the overlap gained)
-  p.pingpong = (n_units > grid && nw == 1) ? 1 : 0;
+  p.pingpong = (n_units > workers && nw == 1) ? 1 : 0;
   p.status = t->status;
-  k_gemm_tc<EPI><<<grid, kGemmThreads, smem, t->s>>>(w0, w1, w2, ma, p, stages);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "GEMM launch failed: %s", cudaGetErrorString(e));
+  cudaError_t e;
+  if (pair) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * workers); cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem; cfg.stream = t->s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, k_gemm_tc<EPI, true>, w0, w1, w2, *ma_half, p, stages);
+  } else {
+    k_gemm_tc<EPI, false><<<workers, kGemmThreads, smem, t->s>>>(w0, w1, w2, ma, p, stages);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return tfail(t, DC_ERR_CUDA, "GEMM launch failed: %s", cudaGetErrorString(e));
+  }
   return DC_OK;
 }
 
@@ -491,9 +525,15 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   const int d = g.d_model, nq = g.n_q_heads, nkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff;
   const int M = m.nv * m.batch * m.R_cap;
   const int BN = pick_bn(M);
-  ActMaps* am = nullptr;
+  ActMaps *am = nullptr, *amh = nullptr;
   int rc = get_act_maps(t, a, BN, &am);
   if (rc != DC_OK) return rc;
+  if (BN % 32 == 0 && BN >= 64 && M > BN) {
+    rc = get_act_maps(t, a, BN / 2, &amh);
+    if (rc != DC_OK) return rc;
+    rc = get_act_maps(t, a, BN, &am);   // (the cache may have been rebuilt)
+    if (rc != DC_OK) return rc;
+  }
   const LayerMaps& L = t->layers[layer];
   GemmParams p{};
   p.M = M; p.BN = BN; p.nq = nq; p.nkv = nkv; p.hd = hd;
@@ -503,7 +543,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 
   hook.begin(DC_STAGE_QKV, 1);
   p.N = (nq + 2 * nkv) * hd; p.K = d; p.nsplit = 1;
-  rc = launch_gemm<GEMM_EPI_QKV>(t, L.wq, L.wk, L.wv, am->a, p, nq + 2 * nkv, kStaticQkv);
+  rc = launch_gemm<GEMM_EPI_QKV>(t, L.wq, L.wk, L.wv, am->a, amh ? &amh->a : nullptr, p, nq + 2 * nkv, kStaticQkv);
   hook.end();
   if (rc != DC_OK) return rc;
 
@@ -517,7 +557,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 
   hook.begin(DC_STAGE_OPROJ, 1);
   p.N = d; p.K = nq * hd; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
-  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.wo, L.wo, L.wo, am->o, p, d / kTileN, kStaticOther);
+  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.wo, L.wo, L.wo, am->o, amh ? &amh->o : nullptr, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
 
@@ -528,13 +568,13 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 
   hook.begin(DC_STAGE_GATEUP, 1);
   p.N = F; p.K = d; p.nsplit = 1;
-  rc = launch_gemm<GEMM_EPI_SWIGLU>(t, L.w_gate, L.w_up, L.w_up, am->a, p, F / kTileN, kStaticOther);
+  rc = launch_gemm<GEMM_EPI_SWIGLU>(t, L.w_gate, L.w_up, L.w_up, am->a, amh ? &amh->a : nullptr, p, F / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_DOWN, 1);
   p.N = d; p.K = F; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
-  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.w_down, L.w_down, L.w_down, am->act, p, d / kTileN, kStaticOther);
+  rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.w_down, L.w_down, L.w_down, am->act, amh ? &amh->act : nullptr, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
 

@@ -64,7 +64,14 @@ __host__ __device__ inline int gemm_stage_bytes(int nw, int BN) {
   return nw * kTileN * kTileK * 2 + BN * kTileK * 2;
 }
 
-template <int EPI>
+// PAIR: the launch uses clusters of two CTAs and every MMA is a pair MMA (cta_group::2, M = 256):
+// the two CTAs own adjacent weight tiles and each stages only half of the activation block, so a
+// k-block is 16 KB of weights plus 16 KB of activations per CTA instead of 16 + 32 - the main
+// loops of these GEMMs are bound by what an SM takes in from L2.  The even CTA issues the MMAs;
+// TMA loads of both CTAs report to its full barrier, tcgen05.commit releases ring slots and
+// signals the accumulators in both; the odd CTA's epilogue warps report the drained accumulators
+// to the even CTA's barrier.  No load is multicast.
+template <int EPI, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a,
@@ -82,9 +89,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   // Column blocks of one weight tile sit next to each other in the unit order, so that the
   // CTAs that share a weight tile run together and all but one read it from L2.
   const int n_cblk = (p.M + p.BN - 1) / p.BN;
-  const int per_split = p.tiles * n_cblk;
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // worker index: CTA or CTA pair
+  const int n_cta = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int a_rows = PAIR ? p.BN / 2 : p.BN;                             // activation rows this CTA stages
+  const int per_split = (PAIR ? p.tiles / 2 : p.tiles) * n_cblk;
   const int n_units = per_split * p.nsplit;
-  const int stage_bytes = gemm_stage_bytes(NW, p.BN);
+  const int stage_bytes = gemm_stage_bytes(NW, a_rows);
   const int KB = p.K / kTileK;
   const bool pp = p.pingpong != 0;
   const uint32_t up_off = pp ? 128u : 256u;   // second accumulator of a set (gate / up), or the odd k-steps' one
@@ -97,6 +108,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     const int rem = u - w.split * per_split;
     w.tile = rem / n_cblk;
     w.cblk = rem - w.tile * n_cblk;
+    if (PAIR) w.tile = 2 * w.tile + (int)rank;
     w.kb0 = (int)(((long long)w.split * KB) / p.nsplit);
     w.nkb = (int)(((long long)(w.split + 1) * KB) / p.nsplit) - w.kb0;
     // which weight matrix and which row of it this tile starts at
@@ -112,7 +124,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int i = 0; i < stages; ++i) { ptx::mbar_init(&bar_full[i], 1); ptx::mbar_init(&bar_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], PAIR ? 256 : 128); }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&map_w0);
     ptx::prefetch_tmap(&map_a);
@@ -127,6 +139,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  if (PAIR) {
+    // both CTAs hold all 512 columns, so the pair MMA's accumulator address names the same columns
+    // in both; the partner's barriers are initialised before any load can report to them
+    if (threadIdx.x == 0 && tmem_base != 0) abort_flag = 1;
+    ptx::cluster_sync();
+  }
 
   // One thread issues every TMA load and one every MMA, so their own instruction streams are on
   // the critical path: slot indices, addresses and descriptors advance by additions only.
@@ -137,31 +155,40 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
       uint32_t s = 0, ph = 0, slot = ring0;
       bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      const uint32_t full_r0 = (PAIR && rank != 0) ? ptx::mapa_shared(full0, 0) : full0;   // the even CTA's
+      for (int u = cta; u < n_units && ok; u += n_cta) {
         const Unit w = unit_of(u);
-        const int arow = w.cblk * p.BN;
+        const int arow = w.cblk * p.BN + (int)rank * a_rows;
         for (int i = 0; i < w.nkb; ++i) {
           if (!ptx::mbar_wait_a(empty0 + 8u * s, ph ^ 1u, &abort_flag)) { ok = false; break; }
-          ptx::mbar_expect_tx_a(full0 + 8u * s, (uint32_t)stage_bytes);
           const int kc = (w.kb0 + i) * kTileK;
-          ptx::tma_load_2d_a(slot, w.map_w, full0 + 8u * s, kc, w.wrow);
-          if (NW == 2) ptx::tma_load_2d_a(slot + kTileN * kTileK * 2, &map_w1, full0 + 8u * s, kc, w.wrow);
-          ptx::tma_load_2d_a(slot + NW * kTileN * kTileK * 2, &map_a, full0 + 8u * s, kc, arow);
+          if (PAIR) {
+            if (rank == 0) ptx::mbar_expect_tx_a(full0 + 8u * s, 2u * (uint32_t)stage_bytes);
+            const uint32_t bar = full_r0 + 8u * s;
+            ptx::tma_load_2d_pair_a(slot, w.map_w, bar, kc, w.wrow);
+            if (NW == 2) ptx::tma_load_2d_pair_a(slot + kTileN * kTileK * 2, &map_w1, bar, kc, w.wrow);
+            ptx::tma_load_2d_pair_a(slot + NW * kTileN * kTileK * 2, &map_a, bar, kc, arow);
+          } else {
+            ptx::mbar_expect_tx_a(full0 + 8u * s, (uint32_t)stage_bytes);
+            ptx::tma_load_2d_a(slot, w.map_w, full0 + 8u * s, kc, w.wrow);
+            if (NW == 2) ptx::tma_load_2d_a(slot + kTileN * kTileK * 2, &map_w1, full0 + 8u * s, kc, w.wrow);
+            ptx::tma_load_2d_a(slot + NW * kTileN * kTileK * 2, &map_a, full0 + 8u * s, kc, arow);
+          }
           if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
         }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      const uint32_t idesc = ptx::idesc_bf16(kTileN, p.BN);
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = ptx::idesc_bf16(PAIR ? 2 * kTileN : kTileN, p.BN);
       const uint32_t ring0 = ptx::smem_u32(smem);
       const uint32_t full0 = ptx::smem_u32(&bar_full[0]), empty0 = ptx::smem_u32(&bar_empty[0]);
       const uint64_t hi = ptx::smem_desc_sw128_hi();
       uint32_t s = 0, ph = 0, slot = ring0;
       bool ok = true;
       int j = 0;   // units of this CTA so far
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++j) {
+      for (int u = cta; u < n_units && ok; u += n_cta, ++j) {
         const Unit w = unit_of(u);
         const uint32_t set = pp ? (uint32_t)(j & 1) : 0u;
         // the epilogue has drained this set (its use before the last one)
@@ -177,6 +204,29 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           const uint64_t dw0 = hi | (uint64_t)(slot >> 4);
           const uint64_t dw1 = dw0 + (kTileN * kTileK * 2 >> 4);
           const uint64_t da = dw0 + (NW * kTileN * kTileK * 2 >> 4);
+          if (PAIR) {
+            if (NW == 2) {
+              ptx::umma_bf16_pair(acc0, dw0, da, idesc, acc_first);
+              ptx::umma_bf16_pair(acc1, dw1, da, idesc, acc_first);
+#pragma unroll
+              for (int kk = 1; kk < kTileK / 16; ++kk) {
+                ptx::umma_bf16_pair_acc(acc0, dw0 + 2 * kk, da + 2 * kk, idesc);
+                ptx::umma_bf16_pair_acc(acc1, dw1 + 2 * kk, da + 2 * kk, idesc);
+              }
+            } else if (pp) {
+              ptx::umma_bf16_pair(acc0, dw0, da, idesc, acc_first);
+              ptx::umma_bf16_pair_acc(acc0, dw0 + 2, da + 2, idesc);
+              ptx::umma_bf16_pair_acc(acc0, dw0 + 4, da + 4, idesc);
+              ptx::umma_bf16_pair_acc(acc0, dw0 + 6, da + 6, idesc);
+            } else {
+              ptx::umma_bf16_pair(acc0, dw0, da, idesc, acc_first);
+              ptx::umma_bf16_pair(acc1, dw0 + 2, da + 2, idesc, acc_first);
+              ptx::umma_bf16_pair_acc(acc0, dw0 + 4, da + 4, idesc);
+              ptx::umma_bf16_pair_acc(acc1, dw0 + 6, da + 6, idesc);
+            }
+            acc_first = 1;
+            ptx::umma_commit_pair_a(empty0 + 8u * s);   // frees the slot in both CTAs
+          } else {
           if (NW == 2) {
             ptx::umma_bf16(acc0, dw0, da, idesc, acc_first);
             ptx::umma_bf16(acc1, dw1, da, idesc, acc_first);
@@ -198,9 +248,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           }
           acc_first = 1;
           ptx::umma_commit_a(empty0 + 8u * s);  // slot free once these MMAs have read it
+          }
           if (++s == (uint32_t)stages) { s = 0; ph ^= 1u; slot = ring0; } else slot += (uint32_t)stage_bytes;
         }
-        if (ok) ptx::umma_commit(&acc_full[set]);   // this unit's accumulators are complete
+        if (ok) {   // this unit's accumulators are complete (in both CTAs of a pair)
+          if (PAIR) ptx::umma_commit_pair(&acc_full[set]);
+          else ptx::umma_commit(&acc_full[set]);
+        }
       }
     }
   } else {
@@ -209,7 +263,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     const int f = quarter * 32 + lane;  // feature (weight row) inside the tile = TMEM lane
     bool ok = true;
     int j = 0;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++j) {
+    const uint32_t acc_empty_r0 = (PAIR && rank != 0) ? ptx::mapa_shared(ptx::smem_u32(&acc_empty[0]), 0) : 0u;
+    for (int u = cta; u < n_units && ok; u += n_cta, ++j) {
       const Unit w = unit_of(u);
       const int tile = w.tile, split = w.split;
       const uint32_t set = pp ? (uint32_t)(j & 1) : 0u;
@@ -328,13 +383,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         }
       }
       }
-      // the set may be overwritten by the unit after the next
+      // the set may be overwritten by the unit after the next; the even CTA's MMA issuer waits
+      // for the epilogue warps of both CTAs
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&acc_empty[set]);
+      if (PAIR && rank != 0) ptx::mbar_arrive_remote(acc_empty_r0 + 8u * set);
+      else ptx::mbar_arrive(&acc_empty[set]);
     }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair leaves while the other may still read its shared memory or signal its
+  // barriers
+  if (PAIR) ptx::cluster_sync();
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, tmem_cols);
