@@ -444,7 +444,7 @@ def main():
 
     peaks = _peaks()
     gemm_ms = sum(stage_ms[n] for n in ("qkv", "oproj", "gateup", "down", "dense"))
-    M = 2 * wl.batch * ((wl.last_len + wl.win_len + 15) // 16 * 16)
+    M = (1 if args.prev == "carried" else 2) * wl.batch * ((wl.last_len + wl.win_len + 15) // 16 * 16)
     w_bytes = 2.0 * _layer_param_count(wl) * n_layers
     flops = 2.0 * _layer_param_count(wl) * n_layers * M
     t_hbm = w_bytes / (peaks["hbm"] * 1e9)

@@ -323,8 +323,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           for (int j = 0; j < 32; ++j) {
             const int m = m_base + c0 + j;
             if (j < width && m < p.M) {
+              // silu(g) = g * (0.5 + 0.5 * tanh(g / 2)): one special-function instruction (as in
+              // the fused chain's epilogue; tanh.approx is good to 2^-11, the result goes to bf16)
               const float g = acc[j];
-              dst[(size_t)m * p.N] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * up[j]);
+              float th;
+              asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * g));
+              dst[(size_t)m * p.N] = __float2bfloat16_rn(g * fmaf(0.5f, th, 0.5f) * up[j]);
             }
           }
         } else {  // GEMM_EPI_QKV
