@@ -44,7 +44,7 @@ def _peaks():
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_dense_chain launch (ncu --set full, 4-layer
 # case, see profiles/dense_chain_llada8b_b1.md) and the hash of the kernel sources it belongs to
 _TRAFFIC = dict(workload="llada8b_b1", dram_bytes_per_layer_launch=469.38e6 + 9.10e6,
-                kernel_sha256="3e2a9ca3d174cdae")
+                kernel_sha256="1b2ff003d0f8861d")
 
 
 def _kernel_hash():
