@@ -358,6 +358,28 @@ static int pick_split(int tiles, int KB, int max_split) {
   return s;
 }
 
+// K splits of a split-K projection on the per-op path.  With few units (one column block) the
+// splits fill the SMs (pick_split).  With many, units come in rounds over the workers (SMs, or SM
+// pairs) and the last round is partly empty - 160 pair-units on 74 pairs are 3 rounds for 2.16
+// rounds of work; splitting K makes the rounds finer at the price of one more fp32 partial array
+// written and read back per split.  Rough model: GEMM at 1 PFLOP/s, partials at 5 TB/s.
+static int pick_split_rounds(const TcState* t, int tiles, int M, int BN, int N, int K, int max_split) {
+  const int n_cblk = (M + BN - 1) / BN;
+  if (n_cblk <= 1) return pick_split(tiles * n_cblk, K / kTileK, max_split);
+  const bool pair = t->gemm_pairs && tiles % 2 == 0 && BN % 32 == 0 && BN >= 64 && t->n_sm >= 2;
+  const int units = (pair ? tiles / 2 : tiles) * n_cblk, workers = pair ? t->n_sm / 2 : t->n_sm;
+  const double t1 = 2.0 * M * N * K / 1e15, work_rounds = (double)units / workers;
+  const double per_split = 2.0 * M * N * 4.0 / 5e12;
+  int best = 1;
+  double best_t = 1e30;
+  for (int s = 1; s <= max_split && (K / kTileK) / s >= 8; ++s) {
+    const double rounds = (double)((units * s + workers - 1) / workers) / s;
+    const double est = t1 * rounds / work_rounds + (s - 1) * per_split;
+    if (est < best_t - 1e-9) { best_t = est; best = s; }
+  }
+  return best;
+}
+
 int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,
                  const __nv_bfloat16* v_cache) {
   const dc_config& g = t->g;
@@ -556,7 +578,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_OPROJ, 1);
-  p.N = d; p.K = nq * hd; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
+  p.N = d; p.K = nq * hd; p.nsplit = pick_split_rounds(t, d / kTileN, M, BN, p.N, p.K, t->max_split);
   rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.wo, L.wo, L.wo, am->o, amh ? &amh->o : nullptr, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
@@ -573,7 +595,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   if (rc != DC_OK) return rc;
 
   hook.begin(DC_STAGE_DOWN, 1);
-  p.N = d; p.K = F; p.nsplit = pick_split((d / kTileN) * ((M + BN - 1) / BN), p.K / kTileK, t->max_split);
+  p.N = d; p.K = F; p.nsplit = pick_split_rounds(t, d / kTileN, M, BN, p.N, p.K, t->max_split);
   rc = launch_gemm<GEMM_EPI_PARTIAL>(t, L.w_down, L.w_down, L.w_down, am->act, amh ? &amh->act : nullptr, p, d / kTileN, kStaticOther);
   hook.end();
   if (rc != DC_OK) return rc;
