@@ -41,18 +41,29 @@ def _peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_dense_chain launch (ncu --set full, 4-layer
-# case, see profiles/dense_chain_llada8b_b1.md) and the hash of the kernel sources it belongs to
-_TRAFFIC = dict(workload="llada8b_b1", dram_bytes_per_layer_launch=469.38e6 + 9.10e6,
-                kernel_sha256="1b2ff003d0f8861d")
-
-
 def _kernel_hash():
     import hashlib
     h = hashlib.sha256()
     for f in ("tc_chain.cuh", "tc_ptx.cuh"):
         h.update(open(os.path.join(ROOT, "paper_2604_15750_b200", "csrc", f), "rb").read())
     return h.hexdigest()[:16]
+
+
+def _traffic_record(workload):
+    """DRAM traffic of one k_dense_chain launch (dram__bytes_read.sum + dram__bytes_write.sum of an
+    ncu capture), read from the tracked summary of that capture: a line
+    `bench-traffic: workload=<name> dram_bytes_per_launch=<bytes> kernel_sha256=<hash>` in
+    profiles/dense_chain_<workload>.md.  None when there is no such line or the kernel sources
+    have changed since the counters were taken."""
+    import re
+    path = os.path.join(ROOT, "profiles", f"dense_chain_{workload}.md")
+    if not os.path.exists(path):
+        return None
+    m = re.search(r"bench-traffic:\s*workload=(\S+)\s+dram_bytes_per_launch=([0-9.eE+]+)\s+kernel_sha256=([0-9a-f]+)",
+                  open(path).read())
+    if not m or m.group(1) != workload or m.group(3) != _kernel_hash():
+        return None
+    return float(m.group(2))
 
 
 def _layer_param_count(wl):
@@ -151,7 +162,7 @@ def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=
                        f"extrapolated to {wl.n_layers} layers, {R} rows, {W} positions, batch {wl.batch}")
 
 
-def _oracle_committed(wl, weights_dev, toks, lens, steer):
+def _oracle_committed(wl, weights_dev, toks, lens, steer, decisions=None):
     """Committed tokens of the full steered step by the oracle's decisions (not timed): the
     steering replaces the stack's output, so this needs the LM head only."""
     from oracle import adapters
@@ -161,22 +172,24 @@ def _oracle_committed(wl, weights_dev, toks, lens, steer):
     ow = adapters.weights_from_torch(one)
     ocfg = adapters.config_from_workload(wl, n_layers=0)
     total = 0
+    per_seq = []
     for b in range(wl.batch):
         Lb, W = lens["last_len"][b], lens["win_len"][b]
         hf = (adapters.to_np(steer[b, 0, :W]), adapters.to_np(steer[b, 1, :W]))
         o = O.step(ocfg, ow, None, None, 0, toks["last_ids"][b, :Lb].numpy(),
                    toks["win_ids"][b, :W].numpy(), lens["remain_len"][b], h_final=hf)
         total += len(o["selected"])
+        per_seq.append(dict(pred=o["pred"], block_len=int(o["block_len"]), selected=list(o["selected"])))
+    if decisions is not None:
+        decisions.extend(per_seq)
     return total
 
 
-def _config(wl, n_layers, **extra):
-    """The workload description both arms print."""
-    c = dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
-             window=wl.win_len, layers=n_layers, variants="curr+prev", steering="decay",
-             l2="inputs larger than L2 (weights streamed every step)")
-    c.update(extra)
-    return c
+def _config(wl, n_layers, variants="curr+prev"):
+    """The workload description; both arms print exactly this."""
+    return dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
+                window=wl.win_len, layers=n_layers, variants=variants, steering="decay",
+                l2="inputs larger than L2 (weights streamed every step)")
 
 
 def _setup(wl, dev, n_layers):
@@ -215,8 +228,9 @@ def run_reference(args, wl, rank, world):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=_config(wl, n_layers, committed_per_step=committed),
-                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                config=_config(wl, n_layers), committed_per_step=committed,
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample,
+                                  extrapolated=True),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
@@ -306,6 +320,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debug: run fewer layers (invalid as a result)")
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-coop", action="store_true",
+                    help="profiling: launch the fused dense kernel without the cooperative attribute "
+                         "(ncu cannot replay cooperative cluster launches); same grid, same work")
     ap.add_argument("--mode", default="step", choices=["step", "generate", "prefill"],
                     help="step: the bench line; generate / prefill: measurements of the decoding "
                          "loop and of dc_prefill on the same model shape (one GPU, own JSON line)")
@@ -348,6 +365,8 @@ def main():
         toks = inputs.make_tokens(wl_r)
         steer = inputs.make_steering(wl_r, weights["lm_head"], profile="decay")
     eng = DepCap.from_workload(wl, weights, n_layers=n_layers, impl=1 if args.kernels == "simt" else 0)
+    if args.no_coop:
+        eng.set_option(1, 0)
     B, W = wl.batch, eng.max_window
     kc, vc = pack_kv_cache(k_log, v_log, eng.max_batch, eng.max_ctx)
     last_h = torch.zeros((B, eng.max_last), dtype=torch.int32).pin_memory()
@@ -443,52 +462,109 @@ def main():
         return
 
     peaks = _peaks()
+    src = peaks["source"] + (" (of measured)" if peaks["source"] == "measured" else " (of fallback)")
+    nv = 1 if args.prev == "carried" else 2
+    Rcap = (wl.last_len + wl.win_len + 15) // 16 * 16
+    M = nv * wl.batch * Rcap
+    fused = launches.get("dense", 0) > 0
+
+    def roof_entry(kernel, ms, nbytes, flops, launches_per_step):
+        """Roofline of one kernel group over a step: the binding resource is the one whose floor
+        (bytes / measured copy bandwidth, flops / measured sustained bf16 rate) is larger."""
+        t_hbm = nbytes / (peaks["hbm"] * 1e9)
+        t_tensor = flops / (peaks["bf16_sustained"] * 1e12)
+        if ms <= 0:
+            return None
+        if t_hbm >= t_tensor:
+            ach = nbytes / (ms * 1e-3) / 1e9
+            r = dict(bound="hbm", achieved=ach, peak=peaks["hbm"], unit="GB/s", frac=ach / peaks["hbm"])
+        else:
+            ach = flops / (ms * 1e-3) / 1e12
+            r = dict(bound="tensor", achieved=ach, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                     frac=ach / peaks["bf16_sustained"])
+        r.update(kernel=kernel, ms_per_step=round(ms, 4), launches_per_step=launches_per_step,
+                 algorithmic_bytes=nbytes, algorithmic_flops=flops, traffic=None, peak_source=src)
+        return r
+
+    # dense layers: every weight byte once per step; 2 flops per parameter and activation row
     gemm_ms = sum(stage_ms[n] for n in ("qkv", "oproj", "gateup", "down", "dense"))
-    M = (1 if args.prev == "carried" else 2) * wl.batch * ((wl.last_len + wl.win_len + 15) // 16 * 16)
     w_bytes = 2.0 * _layer_param_count(wl) * n_layers
-    flops = 2.0 * _layer_param_count(wl) * n_layers * M
-    t_hbm = w_bytes / (peaks["hbm"] * 1e9)
-    t_tensor = flops / (peaks["bf16_sustained"] * 1e12)
-    if t_hbm >= t_tensor:
-        ach = w_bytes / (gemm_ms * 1e-3) / 1e9
-        roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm"], unit="GB/s",
-                    frac=ach / peaks["hbm"])
-    else:
-        ach = flops / (gemm_ms * 1e-3) / 1e12
-        roof = dict(bound="tensor", achieved=ach, peak=peaks["bf16_sustained"], unit="TFLOP/s",
-                    frac=ach / peaks["bf16_sustained"])
-    # DRAM traffic of the dense chain from the ncu capture summarised in
-    # profiles/dense_chain_llada8b_b1.md (one launch = one layer); valid only for the kernel
-    # sources it was taken with and for this workload, scaled to the launches of one step
-    traffic = None
-    if wl.name == _TRAFFIC["workload"] and _kernel_hash() == _TRAFFIC["kernel_sha256"]:
-        per_layer = _TRAFFIC["dram_bytes_per_layer_launch"]
-        first = per_layer * (wl.d_model * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim) / _layer_param_count(wl)
-        traffic = per_layer * n_layers + first
-    roof.update(kernel="k_dense_chain: dense-layer GEMMs (QKV, O, gate/up, down) + norms, all launches of one step",
-                traffic=traffic, peak_source=peaks["source"] + " (of measured)" if peaks["source"] == "measured"
-                else "fallback (of fallback)", stage_ms={k: round(v, 4) for k, v in stage_ms.items()})
+    dense_name = ("k_dense_chain: O projection, norms, gate/up + SwiGLU, down projection, QKV + RoPE of the "
+                  "next layer in one persistent launch per layer" if fused else
+                  "k_gemm_tc: per-op QKV + RoPE, O projection, gate/up + SwiGLU, down projection")
+    roof = roof_entry(dense_name, gemm_ms, w_bytes, w_bytes * M,
+                      sum(launches.get(n, 0) for n in ("qkv", "oproj", "gateup", "down", "dense")))
+    # DRAM traffic of the dense chain from the ncu capture summarised under profiles/ (one launch =
+    # one layer), scaled to the launches of one step (traffic grows with the weights streamed)
+    if fused:
+        per_layer = _traffic_record(wl.name)
+        if per_layer is not None:
+            first = per_layer * (wl.d_model * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim) / _layer_param_count(wl)
+            roof["traffic"] = per_layer * n_layers + first
+    roof["stage_ms"] = {k: round(v, 4) for k, v in stage_ms.items()}
+    # attention: per sequence and layer the context K / V once plus q, k, v, o of the active rows
+    # (both variants); 4 flops per (query row, key, head-dim element)
+    nkv_b = wl.n_kv_heads * wl.head_dim * 2.0
+    att_bytes = sum(n_layers * 2.0 * (P + nv * Rcap) * nkv_b for P in lens["ctx_len"])
+    att_flops = sum(4.0 * n_layers * wl.n_q_heads * wl.head_dim * nv * Rcap * (P + Rcap) for P in lens["ctx_len"])
+    rooflines = [roof,
+                 roof_entry("k_attn: bidirectional block attention, context K / V staged once for both variants",
+                            stage_ms["attn"], att_bytes, att_flops, launches.get("attn", 0)),
+                 roof_entry("k_lmhead_tc + k_lm_combine: LM head with streaming softmax / entropy / KL",
+                            stage_ms["lmhead"], 2.0 * wl.vocab * wl.d_model,
+                            2.0 * (2 * wl.batch * wl.win_len) * wl.vocab * wl.d_model, launches.get("lmhead", 0))]
+    # decision kernels: (5 W + W^2) floats per sequence; at these sizes they are bound by launch
+    # and dependency latency, not by bytes (bench.py --mode decisions gives their bandwidth number)
+    dec_bytes = wl.batch * (5.0 * wl.win_len + wl.win_len ** 2) * 4.0
+    e4, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e4.record(stream)
+    for _ in range(20):
+        eng.select(win_d, lens["win_len"])
+    e5.record(stream)
+    torch.cuda.synchronize()
+    sel_ms = e4.elapsed_time(e5) / 20
+    for name, ms_ in (("k_xlogp: cross log-probs (Eq. 6 halves)", stage_ms["xlogp"]),
+                      ("k_boundary: smoothing, S_k, prefix sums, cut", stage_ms["boundary"]),
+                      ("k_select: CAP-Decoding", sel_ms)):
+        r = roof_entry(name, ms_, dec_bytes, 0.0, 1)
+        if r:
+            r["bound"] = "latency"
+            rooflines.append(r)
+    rooflines = [r for r in rooflines if r]
 
     cpu = None
+    parity = None
     if not args.no_cpu_baseline:
         s = _oracle_sample(inputs.scaled(wl, n_layers=n_layers), weights,
                            k_log, v_log, toks, lens, steer)
-        oc = _oracle_committed(wl, weights, toks, lens, steer)
+        dec = []
+        oc = _oracle_committed(wl, weights, toks, lens, steer, decisions=dec)
         cpu = dict(value=oc / s["est_step_s"], unit=UNIT, cores=torch.get_num_threads(),
                    kind="oracle", sample=s["sample"], est_step_ms=s["est_step_s"] * 1e3,
-                   committed=oc)
+                   committed=oc, extrapolated=True)
+        # the step's decisions against the oracle's on the same steered inputs (rank 0's sequences)
+        pred_g = eng.out["pred_id"][:B].cpu().numpy()
+        blk_g = eng.out["block_len"][:B].cpu().numpy()
+        mask_g = eng.sel["sel_mask"][:B].cpu().numpy()
+        parity = dict(positions=0, pred_mismatch=0, block_len_mismatch=0, subset_mismatch=0)
+        for b, o in enumerate(dec):
+            Wb = lens["win_len"][b]
+            parity["positions"] += Wb
+            parity["pred_mismatch"] += int((pred_g[b, :Wb] != o["pred"]).sum())
+            parity["block_len_mismatch"] += int(int(blk_g[b]) != o["block_len"])
+            parity["subset_mismatch"] += int([i for i in range(Wb) if mask_g[b, i]] != o["selected"])
 
     line = dict(metric=METRIC, value=committed / (ms_step * 1e-3), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=args.warmup, ms_per_step=ms_step, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16" if wl.dtype == "bf16" else "f32",
                 data="synthetic",
-                config=_config(wl, n_layers, committed_per_step=committed, kernels=args.kernels,
-                               **({"variants": "curr + carried prev rows"} if args.prev == "carried" else {}),
-                               status=status_bad),
+                config=_config(wl, n_layers, "curr + carried prev rows" if args.prev == "carried" else "curr+prev"),
+                committed_per_step=committed, kernels=args.kernels, status=status_bad,
                 clocks=clocks,
                 e2e=dict(value=committed_e2e / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
                          h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
-                gpu_launches=gpu_launches, roofline=roof, cpu_baseline=cpu)
+                gpu_launches=gpu_launches, roofline=roof, rooflines=rooflines, cpu_baseline=cpu,
+                decisions_vs_oracle=parity)
     print(json.dumps(line))
     eng.close()
     if dist is not None:

@@ -57,7 +57,9 @@ typedef enum dc_status {
   DC_ERR_NOMEM = 4,       /* workspace allocation failed                                    */
   DC_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                            */
   DC_ERR_TIMEOUT = 6,     /* device side: a bounded wait inside a kernel ran out            */
-  DC_ERR_INDEX = 7        /* device side: a token id outside [0, vocab)                     */
+  DC_ERR_INDEX = 7,       /* device side: a token id outside [0, vocab)                     */
+  DC_ERR_NUMERIC = 8      /* device side: a window position without any finite logit (NaN or  */
+                          /* infinite hidden state); its pred_id is reported as mask_id      */
 } dc_status;
 
 enum { DC_F32 = 0, DC_BF16 = 1 };                       /* dc_config.dtype             */
@@ -309,6 +311,17 @@ typedef struct dc_generate_out {
 } dc_generate_out;
 DC_API int dc_generate(dc_ctx* ctx, const dc_generate_in* in, const dc_generate_out* out);
 
+/* Options of a context.  No paper counterpart.
+ *   DC_OPT_COOPERATIVE (default 1): the fused dense-layer kernel synchronises its CTAs through a
+ *     counter in global memory, which needs all of them resident at once; a cooperative launch
+ *     guarantees that (or fails).  0 launches the same grid without the attribute - for profilers
+ *     that cannot replay cooperative cluster launches.  All CTAs are still resident when the GPU
+ *     runs nothing else, and every wait in the kernel is bounded (DC_ERR_TIMEOUT in status[b]
+ *     otherwise), but the guarantee is gone: not for production use.
+ * Returns DC_ERR_INVALID_ARG for an unknown option. */
+enum { DC_OPT_COOPERATIVE = 1 };
+DC_API int dc_set_option(dc_ctx* ctx, int32_t option, int32_t value);
+
 /* Frees the workspace.  The caller must have synchronised the stream.  Null is a no-op. */
 DC_API int dc_destroy(dc_ctx* ctx);
 
@@ -381,7 +394,7 @@ typedef struct dc_signals_in {
 typedef struct dc_signals_out {   /* device, [batch][max_window]; any but status may be null */
   int32_t* pred_id;
   float *conf, *entropy, *influence, *lse;
-  int32_t* status;                /* [batch], required: DC_OK or DC_ERR_TIMEOUT              */
+  int32_t* status;                /* [batch], required: DC_OK, DC_ERR_TIMEOUT or DC_ERR_NUMERIC */
 } dc_signals_out;
 
 DC_API int dc_signals_static(const dc_signals_in* in, const dc_signals_out* out, void* cuda_stream);

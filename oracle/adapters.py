@@ -21,6 +21,9 @@ def weights_from_torch(wd: dict) -> OracleWeights:
     for lw in wd["layers"]:
         for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm1", "norm2"):
             getattr(w, name).append(to_np(lw[name]))
+        if "bq" in lw:
+            for name in ("bq", "bk", "bv"):
+                getattr(w, name).append(to_np(lw[name]))
     return w
 
 

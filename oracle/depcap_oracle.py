@@ -19,7 +19,7 @@ Diffusion LM Inference"):
 
 The backbone is a black box in the paper; here it is the pre-norm transformer the workload
 configurations name (RMSNorm, rotate-half RoPE, bidirectional attention, grouped KV heads,
-SwiGLU MLP, no biases, untied LM head).
+SwiGLU MLP, untied LM head; no biases, or biases on the q / k / v projections only).
 
 Parity status of each function (what pins it is in tests/test_oracle_*.py):
   forward / attention / rope / rmsnorm / swiglu : pinned (library routines, closed forms)
@@ -86,6 +86,11 @@ class OracleWeights:
     w_down: list = field(default_factory=list)  # [d, F]
     norm1: list = field(default_factory=list)   # [d]
     norm2: list = field(default_factory=list)   # [d]
+    # optional biases of the q / k / v projections (the Dream backbone's attention layers carry
+    # them; LLaDA's do not): per layer [n_q*hd], [n_kv*hd], [n_kv*hd], added before the rotation
+    bq: list = field(default_factory=list)
+    bk: list = field(default_factory=list)
+    bv: list = field(default_factory=list)
     final_norm: np.ndarray | None = None        # [d]
     lm_head: np.ndarray | None = None           # [V, d]
 
@@ -181,9 +186,14 @@ def forward(cfg: OracleConfig, w: OracleWeights, tok: np.ndarray, pos0: int,
     L = cfg.n_layers if n_layers is None else n_layers
     for l in range(L):
         a = _gemm_in(rmsnorm(x, w.norm1[l], cfg.rms_eps), cfg)
-        q = (a @ np.asarray(w.wq[l], dtype=np.float64).T).reshape(R, nq, hd)
-        k = (a @ np.asarray(w.wk[l], dtype=np.float64).T).reshape(R, nkv, hd)
-        v = (a @ np.asarray(w.wv[l], dtype=np.float64).T).reshape(R, nkv, hd)
+        q = a @ np.asarray(w.wq[l], dtype=np.float64).T
+        k = a @ np.asarray(w.wk[l], dtype=np.float64).T
+        v = a @ np.asarray(w.wv[l], dtype=np.float64).T
+        if w.bq:
+            q = q + np.asarray(w.bq[l], dtype=np.float64)
+            k = k + np.asarray(w.bk[l], dtype=np.float64)
+            v = v + np.asarray(w.bv[l], dtype=np.float64)
+        q, k, v = q.reshape(R, nq, hd), k.reshape(R, nkv, hd), v.reshape(R, nkv, hd)
         q = _gemm_in(rope(q, pos, cfg.rope_theta), cfg)
         k = _gemm_in(rope(k, pos, cfg.rope_theta), cfg)
         v = _gemm_in(v, cfg)

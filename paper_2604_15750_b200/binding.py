@@ -13,13 +13,16 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libdepcap.so")
 
 DC_OK = 0
+DC_ERR_TIMEOUT, DC_ERR_INDEX, DC_ERR_NUMERIC = 6, 7, 8
 DC_F32, DC_BF16 = 0, 1
 DC_STEP_INFLUENCE, DC_STEP_BOUNDARY, DC_STEP_EXPORT_KV, DC_STEP_CARRIED_PREV = 1, 2, 4, 8
 DC_IMPL_AUTO, DC_IMPL_SIMT = 0, 1
 STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhead", "xlogp",
                "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
-           "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate", "dc_prefill"]
+           "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate", "dc_prefill",
+           "dc_set_option"]
+DC_OPT_COOPERATIVE = 1
 
 
 class DepCapError(RuntimeError):
@@ -155,6 +158,7 @@ def load_library(path: str | None = None):
     lib_.dc_generate.argtypes = [C.c_void_p, C.POINTER(dc_generate_in),
                                  C.POINTER(dc_generate_out)]
     lib_.dc_destroy.argtypes = [C.c_void_p]
+    lib_.dc_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib_.dc_debug_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
     lib_.dc_last_error.argtypes = [C.c_void_p]
     lib_.dc_last_error.restype = C.c_char_p
@@ -338,12 +342,13 @@ class DepCap:
 
     def step(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len, remain_len,
              influence=True, boundary=True, h_final=None, export_kv=False, carried=None,
-             h_out=None):
+             h_out=None, want_xlogp=True):
         """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled.
         export_kv: also append the last block's K / V to the caches (which are then written)."""
         si, so = self._step_structs(k_cache, v_cache, ctx_len, last_ids, last_len, win_ids,
                                     win_len, remain_len, influence, boundary, h_final,
-                                    export_kv=export_kv, carried=carried, h_out=h_out)
+                                    want_xlogp=want_xlogp, export_kv=export_kv, carried=carried,
+                                    h_out=h_out)
         self._check(self._lib.dc_step(self._ctx, C.byref(si), C.byref(so)))
         return self.out
 
@@ -438,6 +443,11 @@ class DepCap:
                           device=self.device)
         self._check(self._lib.dc_debug_logits(self._ctx, variant, _ptr(out)))
         return out
+
+    def set_option(self, option, value):
+        """dc_set_option (DC_OPT_COOPERATIVE: 0 = launch the fused dense kernel without the
+        cooperative attribute, for profilers)."""
+        self._check(self._lib.dc_set_option(self._ctx, int(option), int(value)))
 
     def synchronize(self):
         self.stream.synchronize()

@@ -310,7 +310,7 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
   if (c->tc_lm) {
     pf.begin(DC_STAGE_LMHEAD, 2);
     int rc = tc_lmhead(c->tc, ml, (const __nv_bfloat16*)h, g.mask_id, g.forbid_mask_pred,
-                       c->ws_pred, c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so);
+                       c->ws_pred, c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so, out->status);
     pf.end();
     if (rc != DC_OK) return fail(c, rc, "tensor-core LM head failed: %s", tc_error(c->tc));
     c->have_logits = false;
@@ -319,13 +319,13 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
     launch_gemm_simt<T>(h, (const T*)c->lm_head, c->logits, Mlm, g.vocab, d, g.vocab,
                         EPI_STORE_F32, s);
     launch_signals_from_logits(c->logits, g.vocab, g.mask_id, g.forbid_mask_pred, ml, c->ws_pred,
-                               c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so, s);
+                               c->ws_conf, c->ws_ent, c->ws_infl, c->ws_lse, so, out->status, s);
     pf.end();
     c->have_logits = true;
   }
   if (out->xlogp) {
     pf.begin(DC_STAGE_XLOGP, 1);
-    launch_xlogp<T>(h, (const T*)c->lm_head, c->ws_pred, c->ws_lse, d, ml, g.max_window,
+    launch_xlogp<T>(h, (const T*)c->lm_head, c->ws_pred, c->ws_lse, d, g.vocab, ml, g.max_window,
                     out->xlogp, s);
     pf.end();
   }
@@ -754,6 +754,15 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
   }
   *out->nfe = nfe;
   return DC_OK;
+}
+
+int dc_set_option(dc_ctx* c, int32_t option, int32_t value) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (option == DC_OPT_COOPERATIVE) {
+    if (c->tc) tc_set_cooperative(c->tc, value != 0);
+    return DC_OK;
+  }
+  return fail(c, DC_ERR_INVALID_ARG, "unknown option %d", option);
 }
 
 int dc_debug_logits(dc_ctx* c, int32_t variant, float* outp) {

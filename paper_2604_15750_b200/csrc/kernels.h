@@ -103,11 +103,11 @@ struct SignalOut {
 void launch_signals_from_logits(const float* logits, int V, int mask_id, int forbid,
                                 const SeqMeta& m, int32_t* ws_pred, float* ws_conf,
                                 float* ws_ent, float* ws_infl, float* ws_lse, SignalOut out,
-                                cudaStream_t s);
+                                int32_t* status, cudaStream_t s);
 
 template <typename T>
 void launch_xlogp(const T* h, const T* lm_head, const int32_t* ws_pred, const float* ws_lse,
-                  int d, const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s);
+                  int d, int V, const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s);
 
 // appends the curr variant's K / V of the last-block rows to one layer's context cache
 // (k_cache / v_cache: that layer's slice); v_ld != 0: v is transposed with that row pitch

@@ -463,7 +463,8 @@ __global__ void __launch_bounds__(256) k_signals(const float* __restrict__ logit
                                                  float* __restrict__ ws_conf,
                                                  float* __restrict__ ws_ent,
                                                  float* __restrict__ ws_infl,
-                                                 float* __restrict__ ws_lse, SignalOut out) {
+                                                 float* __restrict__ ws_lse, SignalOut out,
+                                                 int32_t* __restrict__ status) {
   __shared__ float red[32];
   __shared__ float s_m[8], s_m2[8];
   __shared__ int s_i[8];
@@ -522,6 +523,12 @@ __global__ void __launch_bounds__(256) k_signals(const float* __restrict__ logit
       const float lse2 = mx2 + logf(S2);
       infl = fmaxf(Ad / S - lse + lse2, 0.f);
     }
+    // no finite admissible logit (a NaN / inf hidden row): the argmax sentinel must not reach
+    // the kernels that index the vocabulary matrix with the id
+    if (am < 0 || am >= V || !isfinite(lse)) {
+      am = mask_id;
+      if (status) atomicMax(status + b, (int)DC_ERR_NUMERIC);
+    }
     const int wi = b * m.W_cap + k;
     ws_pred[wi] = am; ws_conf[wi] = conf; ws_ent[wi] = ent; ws_infl[wi] = infl; ws_lse[wi] = lse;
     const int oi = b * out.max_window + k;
@@ -536,9 +543,9 @@ __global__ void __launch_bounds__(256) k_signals(const float* __restrict__ logit
 void launch_signals_from_logits(const float* logits, int V, int mask_id, int forbid,
                                 const SeqMeta& m, int32_t* ws_pred, float* ws_conf,
                                 float* ws_ent, float* ws_infl, float* ws_lse, SignalOut out,
-                                cudaStream_t s) {
+                                int32_t* status, cudaStream_t s) {
   k_signals<<<m.batch * m.W_cap, 256, 0, s>>>(logits, V, mask_id, forbid, m, ws_pred, ws_conf,
-                                              ws_ent, ws_infl, ws_lse, out);
+                                              ws_ent, ws_infl, ws_lse, out, status);
 }
 
 // ---- cross log-probabilities: xlogp[b,i,j] = h_i . W_lm[yhat_j] - lse_i  (Eq. 6 halves) ---------
@@ -546,13 +553,19 @@ template <typename T>
 __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
                                                const T* __restrict__ lm_head,
                                                const int32_t* __restrict__ ws_pred,
-                                               const float* __restrict__ ws_lse, int d, SeqMeta m,
-                                               int max_window, float* __restrict__ xlogp) {
+                                               const float* __restrict__ ws_lse, int d, int V,
+                                               SeqMeta m, int max_window,
+                                               float* __restrict__ xlogp) {
   extern __shared__ __align__(16) float wrow[];  // W_lm[yhat_j] as fp32
   const int b = blockIdx.y, j = blockIdx.x;
   const int W = m.win_len[b];
   if (j >= W) return;
   const int tok = ws_pred[b * m.W_cap + j];
+  if (tok < 0 || tok >= V) {   // never index the vocabulary matrix with an id outside it
+    for (int i = blockIdx.z * (blockDim.x >> 5) + (threadIdx.x >> 5); i < W; i += gridDim.z * (blockDim.x >> 5))
+      if ((threadIdx.x & 31) == 0) xlogp[((size_t)b * max_window + i) * max_window + j] = -INFINITY;
+    return;
+  }
   const T* wr = lm_head + (size_t)tok * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) wrow[i] = to_f<T>(wr[i]);
   __syncthreads();
@@ -592,9 +605,9 @@ __global__ void __launch_bounds__(256) k_xlogp(const T* __restrict__ h,
 
 template <typename T>
 void launch_xlogp(const T* h, const T* lm_head, const int32_t* ws_pred, const float* ws_lse, int d,
-                  const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s) {
+                  int V, const SeqMeta& m, int max_window, float* xlogp, cudaStream_t s) {
   dim3 grid(m.W_cap, m.batch, (m.W_cap + 7) / 8);
-  k_xlogp<T><<<grid, 256, d * sizeof(float), s>>>(h, lm_head, ws_pred, ws_lse, d, m, max_window,
+  k_xlogp<T><<<grid, 256, d * sizeof(float), s>>>(h, lm_head, ws_pred, ws_lse, d, V, m, max_window,
                                                   xlogp);
 }
 
@@ -649,7 +662,7 @@ template void launch_export_kv<__nv_bfloat16>(const __nv_bfloat16*, const __nv_b
   template void launch_swiglu<T>(const float*, int, int, T*, cudaStream_t);                     \
   template void launch_attn_simt<T>(const T*, const T*, const T*, const T*, const T*, int,      \
                                     const SeqMeta&, int, int, int, T*, cudaStream_t);           \
-  template void launch_xlogp<T>(const T*, const T*, const int32_t*, const float*, int,          \
+  template void launch_xlogp<T>(const T*, const T*, const int32_t*, const float*, int, int,     \
                                 const SeqMeta&, int, float*, cudaStream_t);
 DC_INST(float)
 DC_INST(__nv_bfloat16)

@@ -101,11 +101,10 @@ struct TcState {
   int n_sm = 148, lm_stages = 6;
   unsigned int* grid_bar = nullptr;  // arrival counter of the dense chain's grid barrier, then kFlagWords tile flags
   unsigned int qkv_launches = 0;     // chain launches of this step that ran a QKV phase
-  bool balance_qkv = true;
-  bool gemm_pairs = true;            // per-op GEMMs on CTA pairs when there are several column blocks
   unsigned int bar_count = 0;        // arrivals the launches of this step have used up so far
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
-  bool chain_coop = false;           // launched cooperatively (co-residency guaranteed)
+  bool coop_supported = false;       // the device can launch cooperatively
+  bool chain_coop = false;           // the dense chain is launched cooperatively (co-residency guaranteed)
   std::string err;
   bool attrs_set = false;
 };
@@ -266,16 +265,8 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
       if (cudaOccupancyMaxActiveClusters(&n_clusters, k_dense_chain, &cfg) == cudaSuccess &&
           2 * n_clusters >= grid && grid >= 2) {
         t->chain_grid = grid;
-        t->chain_coop = coop != 0;
-        // DC_CHAIN_COOP=0 launches the same grid without the cooperative attribute (all CTAs are
-        // resident anyway when the GPU runs nothing else; every wait in the kernel is bounded).
-        // Profilers that cannot replay cooperative cluster launches need it.
-        const char* e_ = getenv("DC_CHAIN_COOP");
-        if (e_ && e_[0] == '0') t->chain_coop = false;
-        e_ = getenv("DC_BALANCE_QKV");   // DC_BALANCE_QKV=0: every QKV tile by its owner alone
-        if (e_ && e_[0] == '0') t->balance_qkv = false;
-        e_ = getenv("DC_GEMM_PAIRS");    // DC_GEMM_PAIRS=0: per-op GEMMs on single CTAs
-        if (e_ && e_[0] == '0') t->gemm_pairs = false;
+        t->coop_supported = coop != 0;
+        t->chain_coop = t->coop_supported;
       }
     }
     cudaGetLastError();
@@ -310,7 +301,7 @@ static int launch_gemm(TcState* t, const CUtensorMap& w0, const CUtensorMap& w1,
   const int n_cblk = (p.M + p.BN - 1) / p.BN;
   // CTA pairs (each CTA stages half of the activation block) when the shapes allow it and there
   // is more than one column block: below that the fused chain is the path that matters
-  const bool pair = t->gemm_pairs && ma_half != nullptr && tiles % 2 == 0 && p.BN % 32 == 0 &&
+  const bool pair = ma_half != nullptr && tiles % 2 == 0 && p.BN % 32 == 0 &&
                     p.BN >= 64 && n_cblk > 1 && t->n_sm >= 2;
   const int sb = gemm_stage_bytes(nw, pair ? p.BN / 2 : p.BN);
   int stages = (kSmemBudget - static_smem) / sb;
@@ -366,7 +357,7 @@ static int pick_split(int tiles, int KB, int max_split) {
 static int pick_split_rounds(const TcState* t, int tiles, int M, int BN, int N, int K, int max_split) {
   const int n_cblk = (M + BN - 1) / BN;
   if (n_cblk <= 1) return pick_split(tiles * n_cblk, K / kTileK, max_split);
-  const bool pair = t->gemm_pairs && tiles % 2 == 0 && BN % 32 == 0 && BN >= 64 && t->n_sm >= 2;
+  const bool pair = tiles % 2 == 0 && BN % 32 == 0 && BN >= 64 && t->n_sm >= 2;
   const int units = (pair ? tiles / 2 : tiles) * n_cblk, workers = pair ? t->n_sm / 2 : t->n_sm;
   const double t1 = 2.0 * M * N * K / 1e15, work_rounds = (double)units / workers;
   const double per_split = 2.0 * M * N * 4.0 / 5e12;
@@ -411,6 +402,8 @@ void tc_export_kv(TcState* t, int layer, const SeqMeta& m, __nv_bfloat16* k_cach
   launch_export_kv<__nv_bfloat16>(t->k, t->v, t->ldv, m, g.n_kv_heads, g.head_dim, g.max_ctx,
                                   k_cache + (size_t)layer * per_layer, v_cache + (size_t)layer * per_layer, t->s);
 }
+
+void tc_set_cooperative(TcState* t, bool on) { t->chain_coop = on && t->coop_supported; }
 
 bool tc_chain_ok(const TcState* t, const SeqMeta& m) {
   const dc_config& g = t->g;
@@ -470,7 +463,7 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   p.tile_flags = t->grid_bar + 2;
   if (phase_end > CH_QKV) {
     const int tp = (nq + 2 * nkv) / 2, n_help = t->chain_grid / 2 - tp, KB = d / kChainTileK;
-    if (t->balance_qkv && n_help > 0 && tp <= 2 * n_help && nq + 2 * nkv <= kFlagWords && KB >= 4 &&
+    if (n_help > 0 && tp <= 2 * n_help && nq + 2 * nkv <= kFlagWords && KB >= 4 &&
         (size_t)(nq + 2 * nkv) * BN * kChainTile <= (size_t)t->max_split * t->part_stride) {
       // An owner waits for its helper's sums before its own epilogue, so a helper should be done
       // (loop and hand-over) when the owner's loop ends.  Both loops run at the rate an SM takes
@@ -490,16 +483,6 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   }
   p.bar_base = t->bar_count;
   t->bar_count += (unsigned int)(phase_end - phase_begin - 1) * (unsigned int)t->chain_grid;
-#ifdef DC_CHAIN_TRACE
-  static unsigned long long* trace_buf = nullptr;
-  static unsigned long long* trace_dev = nullptr;
-  if (!trace_buf) {
-    trace_buf = (unsigned long long*)malloc(256 * 64 * sizeof(unsigned long long));
-    cudaMalloc(&trace_dev, 256 * 64 * sizeof(unsigned long long));
-  }
-  cudaMemsetAsync(trace_dev, 0, 256 * 64 * sizeof(unsigned long long), t->s);
-  p.trace = trace_dev;
-#endif
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(t->chain_grid); cfg.blockDim = dim3(kChainThreads);
   cfg.dynamicSmemBytes = kChainSmem; cfg.stream = t->s;
@@ -510,27 +493,6 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   attrs[1].val.cooperative = 1;
   cfg.attrs = attrs; cfg.numAttrs = t->chain_coop ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, k_dense_chain, maps, p);
-#ifdef DC_CHAIN_TRACE
-  {
-    static int n_print = 0;
-    if (layer == 5 && n_print < 3) {
-      cudaStreamSynchronize(t->s);
-      cudaMemcpy(trace_buf, trace_dev, 256 * 64 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
-      ++n_print;
-      char fn[256];
-      snprintf(fn, sizeof(fn), "%s/chain_trace_dbg%s_%d.txt", getenv("DC_TRACE_DIR") ? getenv("DC_TRACE_DIR") : ".",
-               getenv("DC_TAG") ? getenv("DC_TAG") : "0", n_print);
-      FILE* f = fopen(fn, "w");
-      if (f) {
-        for (int c = 0; c < t->chain_grid; ++c) {
-          for (int i = 0; i < 64; ++i) fprintf(f, "%llu ", trace_buf[c * 64 + i]);
-          fprintf(f, "\n");
-        }
-        fclose(f);
-      }
-    }
-  }
-#endif
   if (e != cudaSuccess) {
     cudaGetLastError();
     return tfail(t, DC_ERR_CUDA, "dense chain launch failed: %s", cudaGetErrorString(e));
@@ -606,7 +568,7 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 
 int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id, int forbid,
               int32_t* ws_pred, float* ws_conf, float* ws_ent, float* ws_infl, float* ws_lse,
-              SignalOut out) {
+              SignalOut out, int32_t* status) {
   (void)h;  // the tensor map was built over the scheduler's LM-head input buffer
   const dc_config& g = t->g;
   LmParams p;
@@ -621,8 +583,8 @@ int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id,
   k_lmhead_tc<<<groups * nctas, kLmThreads, t->lm_stages * kLmStageBytes + 1024, t->s>>>(t->map_h, t->map_lm,
                                                                                       p, t->lm_stages);
   const int npos = m.batch * m.W_cap;
-  k_lm_combine<<<(npos + 3) / 4, 128, 0, t->s>>>(t->lm_part, nctas, m, ws_pred, ws_conf, ws_ent,
-                                                 ws_infl, ws_lse, out);
+  k_lm_combine<<<(npos + 3) / 4, 128, 0, t->s>>>(t->lm_part, nctas, m, g.vocab, mask_id, status, 1, ws_pred,
+                                                 ws_conf, ws_ent, ws_infl, ws_lse, out);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return tfail(t, DC_ERR_CUDA, "LM-head launch failed: %s", cudaGetErrorString(e));
   return DC_OK;
@@ -777,7 +739,8 @@ extern "C" int dc_signals_static(const dc_signals_in* in, const dc_signals_out* 
   p.ngroups = groups;
   k_lmhead_tc<<<groups * nctas, kLmThreads, sd.lm_stages * kLmStageBytes + 1024, s>>>(map_h, map_lm, p, sd.lm_stages);
   SignalOut so{out->pred_id, out->conf, out->entropy, out->influence, out->lse, in->max_window};
-  k_lm_combine<<<(npos + 3) / 4, 128, 0, s>>>(part, nctas, m, ws_pred, ws_conf, ws_ent, ws_infl, ws_lse, so);
+  k_lm_combine<<<(npos + 3) / 4, 128, 0, s>>>(part, nctas, m, in->vocab, in->mask_id, word, 0, ws_pred, ws_conf,
+                                              ws_ent, ws_infl, ws_lse, so);
   k_static_status<<<1, 32, 0, s>>>(word, out->status, in->batch);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return sfail(DC_ERR_CUDA, cudaGetErrorString(e));

@@ -47,6 +47,8 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
 int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k_cache,
                  const __nv_bfloat16* v_cache);
 
+// Launch the dense chain with (default) or without the cooperative attribute; see DC_OPT_COOPERATIVE.
+void tc_set_cooperative(TcState* t, bool on);
 // true if the persistent dense chain takes this step (all activation rows in one column block)
 bool tc_chain_ok(const TcState* t, const SeqMeta& m);
 // resets the chain's grid barrier; call once at the start of a step
@@ -68,6 +70,6 @@ void tc_export_kv(TcState* t, int layer, const SeqMeta& m, __nv_bfloat16* k_cach
 // the caller's outputs.  Never writes logits.
 int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id, int forbid,
               int32_t* ws_pred, float* ws_conf, float* ws_ent, float* ws_infl, float* ws_lse,
-              SignalOut out);
+              SignalOut out, int32_t* status);
 
 }  // namespace dc

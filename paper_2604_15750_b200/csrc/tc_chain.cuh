@@ -81,9 +81,6 @@ struct ChainParams {
   unsigned int* bar;            // grid barrier arrival counter (counts up over a step)
   unsigned int bar_base;        // its value when this launch starts
   int32_t* status;              // DC_ERR_TIMEOUT lands here; non-zero on entry = do nothing
-#ifdef DC_CHAIN_TRACE
-  unsigned long long* trace;    // [cta][16] globaltimer at phase boundaries (tracing build only)
-#endif
 };
 
 constexpr int kChainThreads = 512;
@@ -94,9 +91,7 @@ constexpr int kChainXch = kChainParts * 128 * kXchRow * 4;  // RoPE exchange buf
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
-#ifndef DC_PREFETCH_AHEAD
-#define DC_PREFETCH_AHEAD 0
-#endif
+// k-blocks of its next unit that a CTA prefetches into L2 when its own loads are issued
 #ifndef DC_PF_GU
 #define DC_PF_GU 4
 #endif
@@ -106,9 +101,7 @@ constexpr int kChainTileK = 64;
 #ifndef DC_PF_QKV
 #define DC_PF_QKV 4
 #endif
-// k-blocks of its next unit that a CTA prefetches into L2 when its own loads are issued
 constexpr int kPfGateUp = DC_PF_GU, kPfDown = DC_PF_DN, kPfQkv = DC_PF_QKV;
-constexpr int kPrefetchAhead = DC_PREFETCH_AHEAD;              // k-blocks the L2 prefetch runs ahead of the TMA loads
 
 struct ChainCtx {
   uint8_t* ring;
@@ -269,15 +262,9 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
   }
 }
 
-#ifdef DC_CHAIN_TRACE
-#define DC_TRACE(slot) p.trace[blockIdx.x * 64 + 16 + (ph) * 4 + (slot)] = ptx::globaltimer()
-#else
-#define DC_TRACE(slot)
-#endif
 
 template <int EPI>
-__device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, const GemmPhase& g,
-                                           const int ph) {
+__device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, const GemmPhase& g) {
   const int BN = p.BN;
   const int half_rows = BN >> 1;  // activation rows this CTA stages (the pair MMA reads both halves)
   ChainItem w;
@@ -295,9 +282,9 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
   };
 
   if (c.warp == 0) {
+    bool ok = true;
     if (c.lane == 0) {
       // ---------------- TMA producer ----------------
-      bool ok = true;
       const uint32_t ring0 = ptx::smem_u32(c.ring);
       const uint32_t full0 = ptx::smem_u32(&c.full[0]), empty0 = ptx::smem_u32(&c.empty[0]);
       const uint32_t full_remote0 = c.rank == 0 ? full0 : ptx::mapa_shared(full0, 0);
@@ -315,23 +302,13 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           const uint32_t par = (c.fill_bits >> ps) & 1u;
           c.fill_bits ^= 1u << ps;
-#ifdef DC_CHAIN_TRACE
-          const long long tw0 = clock64();
-#endif
           ok = ptx::mbar_wait_a(empty0 + 8u * ps, par ^ 1u, c.abort_flag);
-#ifdef DC_CHAIN_TRACE
-          p.trace[blockIdx.x * 64 + 41 + ph * 4] += (unsigned long long)(clock64() - tw0);
-#endif
           if (!ok) break;
           // the bytes of both CTAs are credited to the even CTA's barrier, which its MMA issuer
           // waits on
           if (c.rank == 0) ptx::mbar_expect_tx_a(full0 + 8u * ps, 2u * (uint32_t)slot_bytes);
           const uint32_t bar = full_remote0 + 8u * ps;
           const int kc = kb * kChainTileK;
-          if (kPrefetchAhead > 0 && kb + kPrefetchAhead < w.kb1) {
-            ptx::tma_prefetch_l2_2d(mw, kc + kPrefetchAhead * kChainTileK, wrow);
-            if (nw == 2) ptx::tma_prefetch_l2_2d(mw2, kc + kPrefetchAhead * kChainTileK, wrow2);
-          }
           // weights pass through L2 once (evict first); the activation tile is re-read by every CTA
           // and the small buffers between phases should stay resident (evict last): -5% step time
           ptx::tma_load_2d_pair_hint(pslot, mw, bar, kc, wrow, pol_w);
@@ -340,8 +317,12 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           if (++ps == (uint32_t)stages) { ps = 0; pslot = ring0; } else pslot += (uint32_t)slot_bytes;
         }
       }
-      DC_TRACE(0);
+    }
+    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    {
       // ---------------- L2 prefetch of this CTA's item in the next GEMM phase ----------------
+      // Issued by all lanes of the warp, a k-block each: a prefetch instruction occupies its thread
+      // for a while, and the producer lane is needed again right after the grid barrier.
       ChainItem n;
       if (ok && g.pf_tiles > 0 && chain_item(g.pf_tiles, g.pf_nsplit, g.pf_KB, g.pf_bal_h, n)) {
         const int kb1 = n.kb1 > n.kb0 + g.pf_kb ? n.kb0 + g.pf_kb : n.kb1;
@@ -356,7 +337,7 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
         src(n.tile, m0, r0);
         if (both) { m1 = g.pf_w1; r1 = r0; }
         else if (n.tile2 >= 0) src(n.tile2, m1, r1);
-        for (int kb = n.kb0; kb < kb1; ++kb) {
+        for (int kb = n.kb0 + c.lane; kb < kb1; kb += 32) {
           ptx::tma_prefetch_l2_2d(m0, kb * kChainTileK, r0);
           if (m1 != nullptr) ptx::tma_prefetch_l2_2d(m1, kb * kChainTileK, r1);
         }
@@ -365,58 +346,56 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
   } else if (c.warp == 1) {
     if (c.lane == 0 && c.rank == 0 && has) {
       // ---------------- MMA issuer (even CTA of the pair, for both) ----------------
+      // The issuing thread does not run ahead of the tensor core, so whatever it executes between
+      // two MMAs is added to the MMA period (N = 192: 140 clk per MMA with the descriptors rebuilt
+      // from the slot address every k-block, 97 with this loop; the tensor core's own time is
+      // 96).  The ring is therefore unrolled over its slots: barrier addresses and the low words
+      // of the descriptors of a slot are constants plus loop-invariant registers, the high word
+      // is one constant, and a k-step costs two 32-bit additions.
       const uint32_t idesc = ptx::idesc_bf16(2 * kChainTile, BN);
       bool ok = true;
-      const uint32_t mring0 = ptx::smem_u32(c.ring);
       const uint32_t mfull0 = ptx::smem_u32(&c.full[0]), mempty0 = ptx::smem_u32(&c.empty[0]);
-      const uint64_t desc_hi = ptx::smem_desc_sw128_hi();
-      uint32_t ms = 0, mslot = mring0;
+      const uint32_t hi32 = ptx::smem_desc_hi32();
+      const uint32_t lo0 = ptx::smem_desc_lo(ptx::smem_u32(c.ring));
+      const uint32_t slot16 = (uint32_t)slot_bytes >> 4;
+      constexpr uint32_t kW16 = kChainTile * kChainTileK * 2 >> 4;   // one weight tile in descriptor units
       if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
         ok = ptx::mbar_wait(c.acc_empty, (c.mma_units - 1) & 1u, c.abort_flag);
       }
       ptx::tc_fence_after();
-      uint32_t acc_first = 0;   // 0 until the first k-block of the unit has been issued
-#ifdef DC_CHAIN_TRACE
-      const long long tl0 = clock64();
-#endif
-      for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
-        const uint32_t par = (c.use_bits >> ms) & 1u;
-        c.use_bits ^= 1u << ms;
-#ifdef DC_CHAIN_TRACE
-        const long long tw0 = clock64();
-#endif
-        ok = ptx::mbar_wait_a(mfull0 + 8u * ms, par, c.abort_flag);
-#ifdef DC_CHAIN_TRACE
-        p.trace[blockIdx.x * 64 + 40 + ph * 4] += (unsigned long long)(clock64() - tw0);
-#endif
-        if (!ok) break;
-        const uint64_t dw0 = desc_hi | (uint64_t)(mslot >> 4);
-        const uint64_t dw1 = dw0 + (kChainTile * kChainTileK * 2 >> 4);
-        const uint64_t da = dw0 + ((uint64_t)nw * (kChainTile * kChainTileK * 2 >> 4));
-        if (nw == 2) {
-          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
-          ptx::umma_bf16_pair(c.tmem_base + 256, dw1, da, idesc, acc_first);
+      uint32_t acc = 0;   // 0 until the first k-block of the unit has been issued
+      const uint32_t t0 = c.tmem_base, t1 = c.tmem_base + 256;
+      int kb = w.kb0;
+      while (kb < w.kb1 && ok) {
 #pragma unroll
-          for (int kk = 1; kk < kChainTileK / 16; ++kk) {
-            ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
-            ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
+        for (int s = 0; s < 8; ++s) {
+          if (s < stages && kb < w.kb1) {
+            const uint32_t par = (c.use_bits >> s) & 1u;
+            c.use_bits ^= 1u << s;
+            if (!ptx::mbar_wait_a(mfull0 + 8u * s, par, c.abort_flag)) { ok = false; break; }
+            const uint32_t w0 = lo0 + (uint32_t)s * slot16;
+            const uint32_t a = w0 + (uint32_t)nw * kW16;
+            if (nw == 2) {
+              const uint32_t w1 = w0 + kW16;
+#pragma unroll
+              for (int kk = 0; kk < kChainTileK / 16; ++kk) {
+                ptx::umma_bf16_pair_lo(t0, w0 + 2 * kk, a + 2 * kk, hi32, idesc, kk == 0 ? acc : 1u);
+                ptx::umma_bf16_pair_lo(t1, w1 + 2 * kk, a + 2 * kk, hi32, idesc, kk == 0 ? acc : 1u);
+              }
+            } else {
+              ptx::umma_bf16_pair_lo(t0, w0, a, hi32, idesc, acc);
+              ptx::umma_bf16_pair_lo(t1, w0 + 2, a + 2, hi32, idesc, acc);
+              ptx::umma_bf16_pair_lo(t0, w0 + 4, a + 4, hi32, idesc, 1u);
+              ptx::umma_bf16_pair_lo(t1, w0 + 6, a + 6, hi32, idesc, 1u);
+            }
+            acc = 1;
+            ptx::umma_commit_pair_a(mempty0 + 8u * s);   // frees the slot in both CTAs
+            ++kb;
           }
-        } else {
-          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
-          ptx::umma_bf16_pair(c.tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
-          ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 4, da + 4, idesc);
-          ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw0 + 6, da + 6, idesc);
         }
-        acc_first = 1;
-        ptx::umma_commit_pair_a(mempty0 + 8u * ms);   // frees the slot in both CTAs
-        if (++ms == (uint32_t)stages) { ms = 0; mslot = mring0; } else mslot += (uint32_t)slot_bytes;
       }
-#ifdef DC_CHAIN_TRACE
-      p.trace[blockIdx.x * 64 + 42 + ph * 4] += (unsigned long long)(clock64() - tl0);
-#endif
       if (ok) ptx::umma_commit_pair(c.acc_full);  // both epilogues start
       ++c.mma_units;
-      DC_TRACE(1);
     }
   }
   __syncwarp();
@@ -449,15 +428,6 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
       if (c.lane == 0) got = ptx::flag_wait(p.tile_flags + tile, p.flag_target, c.abort_flag);
       ok = __shfl_sync(0xffffffffu, (int)got, 0) != 0;   // also orders the lanes' loads behind the acquire
     }
-#ifdef DC_CHAIN_TRACE
-    const long long tE0 = clock64();
-    const int eslot = (ph == CH_QKV) ? 13 : 47;   // QKV: 13, 14, 15, 43; gate/up: 47, 51, 55, 59
-    if (threadIdx.x == 64 && (ph == CH_QKV || ph == CH_GATEUP)) p.trace[blockIdx.x * 64 + eslot] = ptx::globaltimer();
-#define DC_ETRACE(c0) if (threadIdx.x == 64 && (ph == CH_QKV || ph == CH_GATEUP)) { const int k_ = ((c0) - col0) / 16; \
-      p.trace[blockIdx.x * 64 + (ph == CH_QKV ? (k_ < 2 ? 14 + k_ : 43) : 51 + 4 * k_)] = (unsigned long long)(clock64() - tE0); }
-#else
-#define DC_ETRACE(c0)
-#endif
     if (ok) {
       ptx::tc_fence_after();
       // 16 columns (activation rows) per step in a rolled loop (the code runs once per unit, so
@@ -520,7 +490,6 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
             for (int k = 0; k < 4; ++k) ha[k] = hn[k];
             rb.c = rn.c; rb.s = rn.s;
           }
-          DC_ETRACE(c0)
         }
         if (kind == ITEM_HELP) {
           __threadfence();
@@ -541,17 +510,14 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
           ptx::tmem_ld_wait();
           chain_emit<EPI>(c, p, g.N, tile, split, f, c0, a0, a1, rb, half);
           rb.c = rn.c; rb.s = rn.s;
-          DC_ETRACE(c0)
         }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(c.acc_empty);
     }
-    if (threadIdx.x == 64) { DC_TRACE(2); }
   }
   // the outputs are read through TMA (async proxy) by other CTAs after the grid barrier
   ptx::fence_proxy_async_global();
-  if (threadIdx.x == 64) { DC_TRACE(3); }
 }
 
 // x[row] += sum of the partial sums (in split order); out[row] = bf16(rmsnorm(x[row]) * g).
@@ -559,8 +525,7 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
 // the partial sums are brought into the (idle) ring by bulk copies, so that a CTA has all of its
 // 160 KB in flight at once instead of a few loads per thread.
 __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, int nsplit,
-                                           const __nv_bfloat16* __restrict__ g, float* red,
-                                           const int ph) {
+                                           const __nv_bfloat16* __restrict__ g, float* red) {
   constexpr int kGrp = kChainThreads / 2;          // threads per row
   const int grp = threadIdx.x / kGrp;              // 0 or 1
   const int t = threadIdx.x - grp * kGrp;          // index inside the group
@@ -584,7 +549,6 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     }
     const bool got = ptx::mbar_wait(c.norm_bar, c.norm_uses & 1u, c.abort_flag);
     ++c.norm_uses;
-    if (threadIdx.x == 0) { DC_TRACE(0); }
     const int row = r0 + grp;
     const bool live = got && row < p.M;
     float* sx = stage + (size_t)grp * narr * d;
@@ -607,7 +571,6 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (c.lane == 0) red[c.warp] = ss;
-    if (threadIdx.x == 0) { DC_TRACE(1); }
     // group-wide exchange: named barriers 5 and 6 (1..4 belong to the QKV epilogue)
     asm volatile("bar.sync %0, %1;" ::"r"(grp + 5), "n"(kGrp) : "memory");
     float tot = 0.f;
@@ -629,7 +592,6 @@ __device__ __forceinline__ void chain_norm(ChainCtx& c, const ChainParams& p, in
     }
     // everyone is done with the staged rows before the next pair is loaded over them
     __syncthreads();
-    if (threadIdx.x == 0) { DC_TRACE(2); }
   }
   ptx::fence_proxy_async_global();  // `a` is the next phase's TMA operand
 }
@@ -687,9 +649,6 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
 
   unsigned int n_barriers = 0;
   for (int ph = p.phase_begin; ph < p.phase_end; ++ph) {
-#ifdef DC_CHAIN_TRACE
-    if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph] = ptx::globaltimer();
-#endif
     GemmPhase g{};
     const bool dead = abort_flag != 0;   // uniform: written before the last CTA-wide barrier
     if (!dead) switch (ph) {
@@ -697,15 +656,15 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         g.w0 = &maps.wo; g.amap = &maps.o; g.tiles = tiles_d; g.nsplit = p.split_o; g.KB = KBq; g.N = p.d;
         g.pf_w0 = &maps.wg; g.pf_w1 = &maps.wu; g.pf_t1 = 0; g.pf_tiles = tiles_f; g.pf_nsplit = 1;
         g.pf_KB = KBd; g.pf_kb = kPfGateUp;
-        chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
+        chain_gemm<CEPI_PARTIAL>(c, p, g);
         break;
       case CH_NORM2:
-        chain_norm(c, p, p.split_o, p.g2, red, ph);
+        chain_norm(c, p, p.split_o, p.g2, red);
         break;
       case CH_GATEUP:
         g.w0 = &maps.wg; g.w1 = &maps.wu; g.amap = &maps.a; g.tiles = tiles_f; g.nsplit = 1; g.KB = KBd; g.N = p.F;
         g.pf_w0 = &maps.wd; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_down; g.pf_KB = KBf; g.pf_kb = kPfDown;
-        chain_gemm<CEPI_SWIGLU>(c, p, g, ph);
+        chain_gemm<CEPI_SWIGLU>(c, p, g);
         break;
       case CH_DOWN:
         g.w0 = &maps.wd; g.amap = &maps.act; g.tiles = tiles_d; g.nsplit = p.split_down; g.KB = KBf; g.N = p.d;
@@ -713,10 +672,10 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
           g.pf_w0 = &maps.wq; g.pf_w1 = &maps.wk; g.pf_w2 = &maps.wv; g.pf_t1 = p.nq; g.pf_t2 = p.nq + p.nkv;
           g.pf_tiles = tiles_qkv; g.pf_nsplit = 1; g.pf_KB = KBd; g.pf_kb = kPfQkv; g.pf_bal_h = p.bal_h;
         }
-        chain_gemm<CEPI_PARTIAL>(c, p, g, ph);
+        chain_gemm<CEPI_PARTIAL>(c, p, g);
         break;
       case CH_NORM1:
-        chain_norm(c, p, p.fold_norm1, p.g1, red, ph);
+        chain_norm(c, p, p.fold_norm1, p.g1, red);
         break;
       default:  // CH_QKV
         g.w0 = &maps.wq; g.w1 = &maps.wk; g.w2 = &maps.wv; g.amap = &maps.a; g.tiles = tiles_qkv;
@@ -724,13 +683,9 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         // attention runs next; meanwhile the O projection of that layer streams into L2 (gate / up
         // of that layer on top of it was measured slower: +2..4% per step for 8..32 k-blocks)
         g.pf_w0 = &maps.wo_n; g.pf_tiles = tiles_d; g.pf_nsplit = p.split_o; g.pf_KB = KBq; g.pf_kb = 64;
-        chain_gemm<CEPI_QKV>(c, p, g, ph);
+        chain_gemm<CEPI_QKV>(c, p, g);
         break;
     }
-#ifdef DC_CHAIN_TRACE
-    __syncthreads();
-    if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 2 * ph + 1] = ptx::globaltimer();
-#endif
     if (ph + 1 < p.phase_end) {
       __syncthreads();
       if (threadIdx.x == 0) {
@@ -754,9 +709,6 @@ k_dense_chain(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     ptx::tmem_dealloc(c.tmem_base, 512);
   }
   if (threadIdx.x == 0 && abort_flag) atomicExch(p.status, DC_ERR_TIMEOUT);
-#ifdef DC_CHAIN_TRACE
-  if (threadIdx.x == 0) p.trace[blockIdx.x * 64 + 12] = ptx::globaltimer();
-#endif
 }
 
 }  // namespace dc

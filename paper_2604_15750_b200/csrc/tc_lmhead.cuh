@@ -152,27 +152,31 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
     float mt = -INFINITY, S = 0.f, A = 0.f, D = 0.f;
     int idx = 0x7fffffff;
     bool ok = true;
-    for (int q = 0; q < my_pairs && ok; ++q) {
+    // Every iteration executes its named barriers whatever happened: a wait that gave up makes
+    // `ok` false for the whole warp and the work is skipped, so that no warp is left waiting on
+    // a barrier the others never reach.
+    for (int q = 0; q < my_pairs; ++q) {
       const int buf = q & 1;
-      ok = ptx::mbar_wait(&acc_full[buf], ((uint32_t)q >> 1) & 1u, &abort_flag);
-      if (!ok) break;
-      ptx::tc_fence_after();
+      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[buf], ((uint32_t)q >> 1) & 1u, &abort_flag));
+      if (ok) ptx::tc_fence_after();
       const int n_in_pair = (2 * q + 1 < my_tiles) ? 2 : 1;
       for (int w = 0; w < n_in_pair; ++w) {
       const int v0 = (slice + (2 * q + w) * nslices) * 128;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float z[32];
-        ptx::tmem_ld_32x32(t_lane + buf * 256 + w * 128 + c * 32, z);
-        ptx::tmem_ld_wait();
+        if (ok) {
+          ptx::tmem_ld_32x32(t_lane + buf * 256 + w * 128 + c * 32, z);
+          ptx::tmem_ld_wait();
+        }
         float* xb = xch[c & 1];
-        if (is_prev) {
+        if (ok && is_prev) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) xb[(row - G) * 33 + i] = z[i];
         }
         if (nv == 2) asm volatile("bar.sync 1, 128;" ::: "memory");
         const int vbase = v0 + c * 32;
-        if (is_curr || is_prev) {
+        if (ok && (is_curr || is_prev)) {
           // chunk maximum over the admissible vocabulary entries
           float cm = -INFINITY;
           int ci = 0x7fffffff;
@@ -207,8 +211,10 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
         }
       }
       }
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(&acc_empty[buf]);
+      if (ok) {
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&acc_empty[buf]);
+      }
     }
     float* rec = p.part + (((size_t)grp * nslices + slice) * 128 + row) * 8;
     rec[0] = mt; rec[1] = __int_as_float(idx); rec[2] = S; rec[3] = A; rec[4] = D;
@@ -223,7 +229,12 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
 }
 
 // Merge the per-CTA records of one window position; one warp per position.
-__global__ void k_lm_combine(const float* __restrict__ part, int nctas, SeqMeta m,
+// A position without any finite admissible logit (a NaN / inf hidden row, or every vocabulary slice
+// gave up in a bounded wait) keeps the argmax sentinel: it is reported as DC_ERR_NUMERIC in
+// status[b * status_stride] and its id is replaced by fallback_id, so that nothing downstream
+// indexes the vocabulary matrix with it.
+__global__ void k_lm_combine(const float* __restrict__ part, int nctas, SeqMeta m, int V,
+                             int fallback_id, int32_t* __restrict__ status, int status_stride,
                              int32_t* __restrict__ ws_pred, float* __restrict__ ws_conf,
                              float* __restrict__ ws_ent, float* __restrict__ ws_infl,
                              float* __restrict__ ws_lse, SignalOut out) {
@@ -284,6 +295,10 @@ __global__ void k_lm_combine(const float* __restrict__ part, int nctas, SeqMeta 
     if (m.nv == 2 && m.have_prev[b]) {
       const float lse2 = mt2 * ln2 + logf(S2);
       infl = fmaxf(D / S - lse + lse2, 0.f);
+    }
+    if (idx < 0 || idx >= V || !isfinite(lse)) {
+      idx = fallback_id;
+      if (status) atomicMax(status + b * status_stride, (int)DC_ERR_NUMERIC);
     }
     const int wi = b * m.W_cap + k;
     ws_pred[wi] = idx; ws_conf[wi] = conf; ws_ent[wi] = ent; ws_infl[wi] = infl; ws_lse[wi] = lse;

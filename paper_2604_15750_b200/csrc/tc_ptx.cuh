@@ -329,6 +329,49 @@ __device__ __forceinline__ void umma_commit_a(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
+// ---- MMA issue with split descriptors ---------------------------------------------------------------
+// The thread that issues tcgen05.mma does not run ahead of the tensor core: every instruction it
+// executes between two MMAs adds its latency to the MMA period (measured: 64 clk per 128x128x16 MMA
+// with the descriptors ready in registers, 107 clk with a dozen address instructions in between,
+// 140 clk at N = 192 when the descriptors are rebuilt from the slot address every k-block).  So
+// issue loops keep the two 32-bit halves of the shared-memory descriptors apart: the upper half is
+// one constant for every tile of this library (swizzle, stride, version), the lower half is the
+// start address, advanced by 32-bit additions of constants; the 64-bit operand is put together
+// inside the asm statement.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) {
+  return (1u << 16) | ((saddr >> 4) & 0x3FFFu);
+}
+__device__ __forceinline__ uint32_t smem_desc_hi32() {
+  return (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+}
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                                  uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// A operand in TMEM (rows = lanes, two bf16 per 32-bit column), B in shared memory
+__device__ __forceinline__ void umma_bf16_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi,
+                                                uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 // constant upper part of smem_desc_sw128; the start address (16-byte units, 14 bits) is added
 __device__ __forceinline__ uint64_t smem_desc_sw128_hi() {
   return ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);

@@ -24,3 +24,17 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """Near-threshold counts and worst errors of every GPU/oracle comparison of the run."""
+    try:
+        import parity
+    except Exception:
+        return
+    if not parity.REPORT:
+        return
+    terminalreporter.write_line("parity against the CPU oracle (near = decisions that differ with the "
+                                "deciding score inside its tolerance; worst = largest errors seen):")
+    for r in parity.REPORT:
+        terminalreporter.write_line(f"  {r['label']}: seqs={r['seqs']} near={r['near']} worst={r['worst']}")

@@ -6,10 +6,15 @@ in the oracle; fp32 path: no rounding):
   logit-like values (lse, xlogp), confidence, entropy : max relative error 2e-2 (bf16) / 1e-4 (f32)
                                                          with denominator max(|ref|, 1)
   influence I_k                                         : 1e-3 absolute where the LM-head inputs
-      are the same bits on both sides (fp32 model, or steered LM-head input): then only the fp32
-      accumulation of the KL sum differs.  Through a bf16 stack the logits themselves differ
-      (they are allowed 2e-2 relative), and I_k, a difference of two log-probability sets,
-      inherits that: 1e-3 + 2e-2 * max_k I_k.
+      are the same bits on both sides (fp32 model, or steered LM-head input) and the logits are
+      accumulated by fp32 FMAs (the CUDA-core LM head): then only the fp32 accumulation of the
+      KL sum differs.  The tensor-core LM head accumulates d_model products per logit in the
+      tensor core's fp32 accumulator, which aligns every product to the running sum and drops the
+      bits below its last place instead of rounding: a logit z comes out low by up to about
+      d_model * 2^-24 * |z| (measured: 2e-4 relative at d_model 4096), and I_k, a difference of
+      logits and log-sum-exps, inherits up to that much of the largest logit:
+      1e-3 + d_model * 2^-24 * max |z|.  Through a bf16 stack the logits themselves differ (they
+      are allowed 2e-2 relative), and I_k inherits that: 1e-3 + 2e-2 * max_k I_k.
 Integer outputs (token ids, block length, selected subset) must be identical unless the deciding
 score lies within the float tolerance of its threshold; those cases are counted and returned.
 """
@@ -141,23 +146,72 @@ def _rel(got, ref):
     return np.abs(got - ref) / np.maximum(np.abs(ref), 1.0)
 
 
-def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
-    """Element-wise comparison; returns counts of near-threshold disagreements."""
+# One record per compare() call; tests/conftest.py prints them in the terminal summary so that the
+# near-threshold counts and the worst errors are visible in a quiet run too.
+REPORT: list[dict] = []
+
+
+def _tc_lmhead(wl):
+    """True when the tensor-core LM head serves this model shape (the library's own rule)."""
+    return wl.dtype == "bf16" and wl.head_dim == 128 and wl.d_model % 128 == 0 and wl.d_ff % 128 == 0
+
+
+def _tc_accumulator_term(wl, o):
+    """What the tensor core's truncating fp32 accumulator may take off the largest logit (see the
+    module docstring); 0 for the CUDA-core LM head."""
+    if not _tc_lmhead(wl):
+        return 0.0
+    zmax = float(np.max(np.abs(o["logits"][np.isfinite(o["logits"])])))
+    if o["logits_prev"] is not None:
+        zmax = max(zmax, float(np.max(np.abs(o["logits_prev"][np.isfinite(o["logits_prev"])]))))
+    return wl.d_model * 2.0 ** -24 * zmax
+
+
+def _score_tolerance(case, o, n, itol, rtol):
+    """How far S_k may move when I_k and H_k move by their own tolerances (itol absolute,
+    rtol * max(H, 1)): smoothing averages, so it does not amplify; dividing by the window maximum
+    (or the max - min range) turns an input error e into at most 2 e / denominator."""
+    hp = case.hyper
+    I, H = o["influence"][:n], o["entropy"][:n]
+    htol = rtol * max(float(np.max(H)), 1.0)
+    if hp.norm_mode == 2:
+        dI = dH = 1.0
+    elif hp.norm_mode == 1:
+        dI = max(float(np.max(I) - np.min(I)), 1e-8)
+        dH = max(float(np.max(H) - np.min(H)), 1e-8)
+    else:
+        dI = max(float(np.max(I)), 1e-8)
+        dH = max(float(np.max(H)), 1e-8)
+    return 2.0 * (itol / dI + hp.lam * htol / dH) + 1e-5
+
+
+def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True, label=None):
+    """Element-wise comparison of one step with the oracle.
+
+    Floats: within the tolerances of the module docstring.  Integers (ids, block length, subset):
+    two checks.  (1) In situ: the oracle's decision rules applied to the GPU's own float outputs
+    must reproduce the GPU's decisions bit for bit - the decision kernels inside the whole step.
+    (2) End to end against the oracle's decisions: identical unless the deciding score of THAT
+    sequence lies within its tolerance of the threshold; such cases are counted in `near`.
+    Returns (near, worst); also appended to REPORT."""
     wl, hp = case.wl, case.hyper
     rtol = rtol if rtol is not None else (1e-4 if wl.dtype == "f32" else 2e-2)
     near = dict(pred=0, block_len=0, subset=0)
-    worst = dict(conf=0.0, entropy=0.0, lse=0.0, influence=0.0, xlogp=0.0)
+    worst = dict(conf=0.0, entropy=0.0, lse=0.0, influence=0.0, influence_tol=0.0, xlogp=0.0,
+                 score_tol=0.0)
     for b, o in ora.items():
         W = case.len["win_len"][b]
         assert gpu["status"][b] == 0
         z = o["logits"]
         # ---- token ids: identical unless the top-2 logits are within tolerance
+        near_pos = []
         for k in range(W):
             gp, op = int(gpu["pred_id"][b, k]), int(o["pred"][k])
             if gp != op:
                 gap = z[k, op] - z[k, gp]
                 assert gap <= rtol * max(1.0, abs(z[k, op])), (b, k, gp, op, gap)
                 near["pred"] += 1
+                near_pos.append(k)
         same = gpu["pred_id"][b, :W] == o["pred"]
         for name in ("conf", "entropy", "lse"):
             # conf/entropy/lse depend on the whole distribution, not on which of two near-tied
@@ -168,7 +222,10 @@ def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
         e = np.abs(gpu["influence"][b, :W] - o["influence"]).max()
         worst["influence"] = max(worst["influence"], float(e))
         same_inputs = wl.dtype == "f32" or case.steer is not None
-        itol = 1e-3 if same_inputs else 1e-3 + rtol * float(np.max(o["influence"]))
+        itol = 1e-3 + _tc_accumulator_term(wl, o)
+        if not same_inputs:
+            itol += rtol * float(np.max(o["influence"]))
+        worst["influence_tol"] = max(worst["influence_tol"], itol)
         assert e <= itol, ("influence", b, e, itol)
         xg, xo = gpu["xlogp"][b, :W, :W], o["xlogp"]
         cols = np.where(same)[0]
@@ -179,35 +236,48 @@ def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
             worst["xlogp"] = max(worst["xlogp"], float(e))
             assert e <= rtol, ("xlogp", b, e)
         # ---- block length
+        have_prev = o["logits_prev"] is not None
         if check_boundary and len(o["score"]):
-            # The score divides I and H by their window maxima, so an input error dI becomes
-            # dI / max(I) in the score (random-init weights give I ~ 1e-5, where fp32 rounding of
-            # the KL sum is already visible).  Bound the score error by the observed input errors.
             n = len(o["score"])
-            dI = np.abs(gpu["influence"][b, :n] - o["influence"][:n]).max()
-            dH = np.abs(gpu["entropy"][b, :n] - o["entropy"][:n]).max()
-            Imax = max(float(np.max(o["influence"][:n])), 1e-8)
-            Hmax = max(float(np.max(o["entropy"][:n])), 1e-8)
-            if hp.norm_mode == 2:
-                Imax = Hmax = 1.0
-            sbound = 4.0 * (dI / Imax + hp.lam * dH / Hmax) + 1e-5
             Lg, Lo = int(gpu["block_len"][b]), int(o["block_len"])
-            if Lg != Lo:
-                lo, hi = min(Lg, Lo), max(Lg, Lo)
-                s_ = o["score"][:hi + 1]
-                assert np.abs(s_[lo:]).min() <= sbound or \
-                    np.abs(o["cum_score"][lo:hi + 1]).min() <= sbound * max(1, hi), (b, Lg, Lo)
-                near["block_len"] += 1
-            elif o["influence"][:n].max() > 0:
-                assert np.abs(gpu["score"][b, :n] - o["score"]).max() <= sbound, \
-                    (b, np.abs(gpu["score"][b, :n] - o["score"]).max(), sbound)
+            # (1) in situ: the boundary rule on the GPU's own I_k, H_k, bit for bit
+            Li, si, ci, csi = O.boundary(gpu["influence"][b, :W], gpu["entropy"][b, :W], W,
+                                         case.len["remain_len"][b], have_prev, case.ocfg)
+            assert Li == Lg, ("block_len in situ", b, Lg, Li)
+            assert np.array_equal(si, gpu["score"][b, :n]), ("score in situ", b)
+            assert np.array_equal(ci, gpu["cum_influence"][b, :n]), ("cum_influence in situ", b)
+            assert np.array_equal(csi, gpu["cum_score"][b, :n]), ("cum_score in situ", b)
+            # (2) against the oracle's own decision
+            if have_prev:
+                stol = _score_tolerance(case, o, n, itol, rtol)
+                worst["score_tol"] = max(worst["score_tol"], stol)
+                cum = hp.boundary_mode == 1
+                dec_o = o["cum_score"] if cum else o["score"]
+                dec_g = gpu["cum_score"][b, :n] if cum else gpu["score"][b, :n]
+                if Lg != Lo:
+                    # the first position where the two sides disagree on "negative" decides
+                    flips = np.where((dec_o < 0) != (dec_g < 0))[0]
+                    assert len(flips), (b, Lg, Lo)
+                    kd = int(flips[0])
+                    assert abs(float(dec_o[kd])) <= stol * ((kd + 1) if cum else 1), \
+                        ("block_len", b, Lg, Lo, kd, float(dec_o[kd]), stol)
+                    near["block_len"] += 1
+                else:
+                    e = np.abs(gpu["score"][b, :n] - o["score"]).max()
+                    assert e <= stol, ("score", b, e, stol)
+            else:
+                assert Lg == Lo, (b, Lg, Lo)
         # ---- selected subset
         cnt = int(gpu["sel_count"][b])
         sel_g = sorted(int(i) for i in gpu["sel_idx"][b, :cnt])
         assert sel_g == [i for i in range(W) if gpu["sel_mask"][b, i]]
-        # the oracle's subset for the GPU's block length (the subset depends on it)
         Lsel = int(gpu["block_len"][b])
         masked = case.win_ids[b, :W].numpy() == wl.mask_id
+        # (1) in situ: Algorithm 1 on the GPU's own c_i and cross log-probs, bit for bit
+        sel_i = O.cap_select(gpu["conf"][b, :W], masked, gpu["xlogp"][b, :W, :W], Lsel, hp.tau_low,
+                             hp.tau_high, hp.gamma, hp.cap_mode)
+        assert sel_g == sel_i, ("subset in situ", b, sel_g, sel_i)
+        # (2) against the oracle's subset for the same block length (the subset depends on it)
         sel_o = O.cap_select(o["conf"], masked, o["xlogp"], Lsel, hp.tau_low, hp.tau_high,
                              hp.gamma, hp.cap_mode)
         if sel_g != sel_o:
@@ -218,10 +288,69 @@ def compare(case: Case, gpu: dict, ora: dict, rtol=None, check_boundary=True):
             close_gamma = np.abs(D[np.isfinite(D)] - hp.gamma).min() <= 2 * rtol
             cs = np.sort(c)
             close_sort = len(cs) > 1 and (np.diff(cs) / np.maximum(cs[1:], 1e-30)).min() <= rtol
-            assert close_tau or close_gamma or close_sort or near["pred"] > 0, (b, sel_g, sel_o)
+            # a near-tied id inside this sequence's block changes a column of its D matrix
+            tied_id = any(k < Lsel for k in near_pos)
+            assert close_tau or close_gamma or close_sort or tied_id, (b, sel_g, sel_o)
             near["subset"] += 1
         # structural checks that hold whatever the rounding did
         assert all(masked[i] and i < Lsel for i in sel_g)
         if masked[:Lsel].any():
             assert cnt >= 1
+    REPORT.append(dict(label=label or wl.name, seqs=len(ora), near=dict(near),
+                       worst={k: float(f"{v:.3g}") for k, v in worst.items()}))
     return near, worst
+
+
+def lm_stage_strict(case: Case, eng, seqs=None):
+    """The LM-head stage alone at the strict tolerances, on rows a real stack produced.
+
+    Three GPU steps on the case's inputs: (A) the last block masked, one variant: its h_out rows
+    are the prev variant's LM-head inputs; (B) one variant with the last block decoded and A's
+    rows carried in as p_prev: the LM head of B sees exactly (h_out of B, h_out of A), both known
+    bit for bit; (C) the ordinary two-variant step.  The oracle's signals on those same rows must
+    match B: ids identical up to near-ties, c / H / lse within rtol, I_k within 1e-3 absolute plus
+    the tensor-core accumulator term (tiny on these rows: random-init logits are below 1).  Returns the worst errors of B against the oracle
+    and the largest |I_k(C) - I_k(B)| (what running both variants in one pass changes)."""
+    wl = case.wl
+    rtol = 2e-2
+    di = case.device_inputs(eng)
+    di.pop("h_final")
+    B, MW, d = wl.batch, eng.max_window, wl.d_model
+    dev = eng.device
+    mask_last = torch.full_like(di["last_ids"], wl.mask_id)
+    hA = torch.zeros((B, MW, d), dtype=wl.torch_dtype, device=dev)
+    eng.step(**{**di, "last_ids": mask_last}, influence=False, boundary=False, h_out=hA)
+    hB = torch.zeros_like(hA)
+    outB = {k: v.clone() for k, v in
+            eng.step(**di, boundary=False, carried=(hA, di["win_len"]), h_out=hB).items()}
+    outC = {k: v.clone() for k, v in eng.step(**di, influence=True, boundary=False).items()}
+    eng.synchronize()
+    worst = dict(conf=0.0, entropy=0.0, lse=0.0, influence=0.0, influence_two_variant=0.0, near_pred=0)
+    for b in (range(B) if seqs is None else seqs):
+        W = case.len["win_len"][b]
+        hc = adapters.to_np(hB[b, :W].cpu())
+        hp_ = adapters.to_np(hA[b, :W].cpu())
+        z = O.logits_of(hc, case.ow.lm_head, case.ocfg)
+        zp = O.logits_of(hp_, case.ow.lm_head, case.ocfg)
+        pred, conf, ent, infl, lse, _ = O.signals_from_logits(z, zp)
+        g = {k: outB[k][b, :W].cpu().numpy() for k in ("pred_id", "conf", "entropy", "influence", "lse")}
+        for k in range(W):
+            if int(g["pred_id"][k]) != int(pred[k]):
+                gap = z[k, pred[k]] - z[k, int(g["pred_id"][k])]
+                assert gap <= rtol * max(1.0, abs(z[k, pred[k]])), (b, k, gap)
+                worst["near_pred"] += 1
+        for name, ref in (("conf", conf), ("entropy", ent), ("lse", lse)):
+            e = float(_rel(g[name], ref).max())
+            worst[name] = max(worst[name], e)
+            assert e <= rtol, (name, b, e)
+        e = float(np.abs(g["influence"] - infl).max())
+        worst["influence"] = max(worst["influence"], e)
+        itol = 1e-3 + _tc_accumulator_term(wl, dict(logits=z, logits_prev=zp))
+        worst["influence_tol"] = max(worst.get("influence_tol", 0.0), itol)
+        assert e <= itol, ("influence, LM-head stage", b, e, itol)
+        e2 = float(np.abs(outC["influence"][b, :W].cpu().numpy() - g["influence"]).max())
+        worst["influence_two_variant"] = max(worst["influence_two_variant"], e2)
+    REPORT.append(dict(label=(wl.name + " / LM-head stage on stack rows"), seqs=B,
+                       near=dict(pred=worst["near_pred"]),
+                       worst={k: float(f"{v:.3g}") for k, v in worst.items() if k != "near_pred"}))
+    return worst

@@ -67,6 +67,31 @@ def test_full_vocabulary_lm_head_signals_and_decisions_match_the_oracle():
     eng.close()
 
 
+def test_influence_tolerance_tensor_core_accumulator_against_fp32_fma():
+    """The same steered LM-head inputs (d_model 4096, logits up to about 15) through both LM heads:
+    the CUDA-core one accumulates each logit with fp32 FMAs and must hold I_k to 1e-3 absolute; the
+    tensor-core one is allowed the accumulator term d_model * 2^-24 * max |z| on top (its fp32
+    accumulator drops the bits of every product below the running sum's last place)."""
+    wl = inputs.scaled(LLADA, n_layers=1, vocab=8192, ctx_min=64, ctx_max=64, batch=2, win_len=128)
+    case = Case(wl, steer="decay")
+    errs = {}
+    for impl in (1, 0):
+        eng = case.make_engine(impl=impl)
+        gpu = case.run_gpu(eng)
+        eng.close()
+        ora = case.run_oracle()
+        errs[impl] = max(float(np.abs(gpu["influence"][b, :wl.win_len] - ora[b]["influence"]).max())
+                         for b in range(wl.batch))
+    zmax = max(float(np.abs(ora[b]["logits"][np.isfinite(ora[b]["logits"])]).max()) for b in range(wl.batch))
+    assert errs[1] <= 1e-3, errs                                   # fp32 FMA accumulation
+    assert errs[0] <= 1e-3 + wl.d_model * 2.0 ** -24 * zmax, (errs, zmax)
+    import parity
+    parity.REPORT.append(dict(label="I_k error, same steered inputs: CUDA-core vs tensor-core LM head",
+                              seqs=wl.batch, near={}, worst=dict(cuda_core=float(f"{errs[1]:.3g}"),
+                                                                 tensor_core=float(f"{errs[0]:.3g}"),
+                                                                 max_logit=float(f"{zmax:.3g}"))))
+
+
 def test_whole_32_layer_step_properties():
     """The benchmark's configuration itself: outputs are finite and in range, the step is
     reproducible bit for bit, the status word is clean."""

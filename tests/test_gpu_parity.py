@@ -136,6 +136,36 @@ def test_out_of_range_token_id_sets_the_status_word():
     eng.close()
 
 
+@pytest.mark.parametrize("tc", [False, True])
+def test_non_finite_hidden_row_sets_the_status_word_and_keeps_the_id_in_range(tc):
+    """A NaN LM-head input row (made on the host) has no finite logit: its argmax is undefined.
+    The step must say so in status[b] and report an id inside the vocabulary (mask_id) instead of
+    the argmax sentinel, which the cross log-prob kernel would otherwise use as a row index.
+    Runs without the cross log-probs first, then with them; both CUDA-core and tensor-core LM head."""
+    wl = inputs.Workload("nan_row", 1, 256, 2, 2, 128, 256, 3000, "bf16", 3, 32, 64, 16, 32, 64, 99) \
+        if tc else SMALL_BF16
+    case = Case(wl, steer="decay")
+    eng = case.make_engine()
+    di = case.device_inputs(eng)
+    di["h_final"][1, 0, 5, :] = float("nan")
+    for want in (False, True):
+        eng.step(**di, want_xlogp=want)
+        eng.synchronize()
+        st = eng.out["status"].cpu().numpy()
+        assert st[1] == 8 and st[0] == 0 and st[2] == 0
+        pred = eng.out["pred_id"].cpu().numpy()
+        assert pred[1, 5] == wl.mask_id
+        for b in range(wl.batch):
+            w = case.len["win_len"][b]
+            assert ((pred[b, :w] >= 0) & (pred[b, :w] < wl.vocab)).all()
+    # the context stays usable and clean inputs give a clean status
+    clean = case.device_inputs(eng)
+    eng.step(**clean)
+    eng.synchronize()
+    assert int(eng.out["status"].abs().max()) == 0
+    eng.close()
+
+
 def test_create_rejects_bad_configurations():
     case = Case(SMALL_BF16)
     with pytest.raises(DepCapError):

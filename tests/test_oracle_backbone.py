@@ -181,3 +181,42 @@ def test_forward_bf16_mode_rounds_only_gemm_inputs():
 def test_swiglu_matches_torch_silu():
     x = np.linspace(-8, 8, 101)
     assert np.allclose(O.silu(x), F.silu(torch.from_numpy(x)).numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_forward_with_qkv_biases_matches_transformers_qwen2():
+    """Biases on the q / k / v projections (none on the output projection), added before the
+    rotation: the attention layers of the Qwen2 family, which the Dream backbone comes from."""
+    from transformers import Qwen2Config, Qwen2Model
+    cfg = Qwen2Config(vocab_size=97, hidden_size=32, intermediate_size=48, num_hidden_layers=2,
+                      num_attention_heads=4, num_key_value_heads=2, rms_norm_eps=1e-5,
+                      rope_theta=10000.0, max_position_embeddings=256, use_sliding_window=False)
+    cfg._attn_implementation = "eager"
+    torch.manual_seed(1)
+    m = Qwen2Model(cfg).double().eval()
+    with torch.no_grad():
+        for n, p in m.named_parameters():
+            if "norm" in n:
+                p.copy_(1.0 + 0.1 * torch.randn_like(p))
+            if n.endswith("proj.bias"):
+                p.copy_(0.5 * torch.randn_like(p))
+    w = _oracle_weights_from_hf(m)
+    sd = {k: v.detach().numpy() for k, v in m.state_dict().items()}
+    for l in range(2):
+        w.bq.append(sd[f"layers.{l}.self_attn.q_proj.bias"])
+        w.bk.append(sd[f"layers.{l}.self_attn.k_proj.bias"])
+        w.bv.append(sd[f"layers.{l}.self_attn.v_proj.bias"])
+    assert f"layers.0.self_attn.o_proj.bias" not in sd
+    ocfg = O.OracleConfig(n_layers=2, d_model=32, n_q_heads=4, n_kv_heads=2, head_dim=8,
+                          d_ff=48, vocab=97, mask_id=96)
+    R, pos0 = 10, 5
+    ids = torch.randint(0, 97, (1, R))
+    with torch.no_grad():
+        want = m(input_ids=ids, attention_mask=torch.zeros(1, 1, R, R, dtype=torch.float64),
+                 position_ids=torch.arange(pos0, pos0 + R)[None]).last_hidden_state[0].numpy()
+    x = O.forward(ocfg, w, ids[0].numpy(), pos0, None, None)
+    got = O.rmsnorm(x, w.final_norm, 1e-5)
+    assert np.allclose(got, want, rtol=1e-5, atol=1e-6)
+    # and the biases matter: without them the result is far off
+    w.bq, w.bk, w.bv = [], [], []
+    x0 = O.forward(ocfg, w, ids[0].numpy(), pos0, None, None)
+    assert np.abs(O.rmsnorm(x0, w.final_norm, 1e-5) - want).max() > 1e-2

@@ -7,9 +7,10 @@ allocates a workspace, so such a caller cannot use dc_step; this entry point kee
 in a fixed array inside the library image instead.
 
 The check: on the same LM-head inputs its outputs equal those dc_step writes (same kernels, same
-tiling), on two calls in a row - the second call runs over the first call's leftovers in the shared
-scratch array, which is exactly the situation the entry point has to handle.  The file sorts last
-so that a run that stops at the first failure has already run every other test.
+tiling) and agree with the CPU oracle's signals for those inputs, on two calls in a row - the
+second call runs over the first call's leftovers in the shared scratch array, which is exactly the
+situation the entry point has to handle - and the free device memory does not move across a call.
+The file sorts last so that a run that stops at the first failure has already run every other test.
 """
 import numpy as np
 import pytest
@@ -35,6 +36,7 @@ def test_static_scratch_entry_matches_dc_step_twice_in_a_row():
     di = case.device_inputs(eng)
     ref = {k: v.clone() for k, v in eng.step(**di).items()}
     eng.synchronize()
+    ora = case.run_oracle()                      # the CPU oracle on the same LM-head inputs
     B, W = case.wl.batch, eng.max_window
     lm_head = eng._weights["lm_head"]
     dev = lm_head.device
@@ -48,8 +50,12 @@ def test_static_scratch_entry_matches_dc_step_twice_in_a_row():
             other = dict(out, **{k: v.clone() for k, v in out.items()})
             signals_static(lm_head, torch.flip(di["h_final"], dims=[2]).contiguous(),
                            [W, W, W], other, mask_id=case.wl.mask_id)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info(dev)[0]
         signals_static(lm_head, di["h_final"], di["win_len"], out, mask_id=case.wl.mask_id)
         torch.cuda.synchronize()
+        if call == 1:    # (the first call on a device may load the kernels' code)
+            assert torch.cuda.mem_get_info(dev)[0] == free_before
         assert out["status"].cpu().tolist() == [0] * B
         for b in range(B):
             w = di["win_len"][b]
@@ -59,6 +65,17 @@ def test_static_scratch_entry_matches_dc_step_twice_in_a_row():
                 assert (np.abs(g - r) / np.maximum(np.abs(r), 1.0)).max() <= tol, (call, name, b)
             g, r = out["influence"][b, :w].cpu().numpy(), ref["influence"][b, :w].cpu().numpy()
             assert np.abs(g - r).max() <= 1e-3, (call, b)
+            # against the oracle: ids identical (steered inputs leave no near-ties here), floats
+            # within the tolerances of the parity tests
+            o = ora[b]
+            assert np.array_equal(out["pred_id"][b, :w].cpu().numpy(), o["pred"]), (call, b)
+            for name, key in (("conf", "conf"), ("entropy", "entropy"), ("lse", "lse")):
+                g = out[name][b, :w].cpu().numpy()
+                assert (np.abs(g - o[key]) / np.maximum(np.abs(o[key]), 1.0)).max() <= 2e-2, (call, name, b)
+            have_prev = case.len["last_len"][b] > 0
+            g = out["influence"][b, :w].cpu().numpy()
+            if have_prev:
+                assert np.abs(g - o["influence"]).max() <= 1e-3, (call, b)
             # positions beyond the window are not written
             assert int(out["pred_id"][b, w:].max().item() if w < W else -7) == -7
     eng.close()
