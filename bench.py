@@ -118,7 +118,7 @@ class ClockSampler:
         return out
 
 
-def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=16, budget_s=None):
+def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=16, budget_s=None, prompt=None):
     """Times the CPU oracle, as it stands, on a bounded sample of the step for sequence 0:
     one transformer layer (curr and prev variants) over the first n_rows active rows and the LM
     head + signals on the first n_head_pos window positions; the full-step time is extrapolated
@@ -140,6 +140,10 @@ def _oracle_sample(wl, weights_dev, k_log, v_log, toks, lens, steer, n_head_pos=
         n_head_pos = max(2, min(n_head_pos, int(n_head_pos * frac)))
     kc = adapters.to_np(k_log[:1, 0]) if k_log is not None else None
     vc = adapters.to_np(v_log[:1, 0]) if v_log is not None else None
+    if prompt is not None and P > 0:
+        # the context cache of the sampled layer from the oracle's own prefill of the prompt (an
+        # input of the step: not timed)
+        kc, vc = O.prefill(ocfg, ow, prompt[0, :P].numpy(), n_layers=1)
     last = toks["last_ids"][0, :Lb].numpy()
     win = toks["win_ids"][0, :W].numpy()
     tok_curr = np.concatenate([last, win]).astype(np.int64)
@@ -185,16 +189,18 @@ def _oracle_committed(wl, weights_dev, toks, lens, steer, decisions=None):
     return total
 
 
-def _config(wl, n_layers, variants="curr+prev"):
+def _config(wl, n_layers, variants="curr+prev", ctx="prefill"):
     """The workload description; both arms print exactly this."""
     return dict(workload=wl.name, batch=wl.batch, ctx=wl.ctx_max, last_block=wl.last_len,
                 window=wl.win_len, layers=n_layers, variants=variants, steering="decay",
+                context=("K / V of the seeded prompt made by the model's own bidirectional prefill"
+                         if ctx == "prefill" else "seeded N(0,1) K / V"),
                 l2="inputs larger than L2 (weights streamed every step)")
 
 
-def _setup(wl, dev, n_layers):
+def _setup(wl, dev, n_layers, noise_ctx=True):
     weights = inputs.make_weights(wl, device=dev, n_layers=n_layers)
-    k_log, v_log = inputs.make_ctx_kv(wl, device=dev, n_layers=n_layers)
+    k_log, v_log = inputs.make_ctx_kv(wl, device=dev, n_layers=n_layers) if noise_ctx else (None, None)
     toks = inputs.make_tokens(wl)
     lens = {k: [int(x) for x in v] for k, v in inputs.make_lengths(wl).items()}
     steer = inputs.make_steering(wl, weights["lm_head"], profile="decay")
@@ -218,7 +224,8 @@ def run_reference(args, wl, rank, world):
     sample = None
     budget = 150.0 / (args.warmup + args.steps)      # the whole run ends within a few minutes
     for i in range(args.warmup + args.steps):
-        s = _oracle_sample(wl1, weights, k_log, v_log, toks, lens, steer, budget_s=budget)
+        s = _oracle_sample(wl1, weights, k_log, v_log, toks, lens, steer, budget_s=budget,
+                           prompt=toks["prompt"] if args.ctx == "prefill" else None)
         sample = s["sample"]
         if i >= args.warmup:
             times.append(s["est_step_s"])
@@ -228,7 +235,7 @@ def run_reference(args, wl, rank, world):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=_config(wl, n_layers), committed_per_step=committed,
+                config=_config(wl, n_layers, ctx=args.ctx), committed_per_step=committed,
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample,
                                   extrapolated=True),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
@@ -310,6 +317,67 @@ def run_prefill(args, wl, dev):
     eng.close()
 
 
+def run_decisions(args, wl, dev):
+    """The decision kernels alone over 8192 synthetic sequences with windows of 128 positions
+    (dc_boundary_batched, dc_select_batched: device-side length arrays): at the sizes of a step
+    they are bound by launch and dependency latency, here their memory traffic is large enough to
+    time.  Algorithmic bytes: boundary 2 W floats in, 3 W floats + 1 int out per sequence; select
+    W floats + W ints + W^2 floats + 1 int in, W bytes + W ints + 1 int out."""
+    import numpy as np
+    from paper_2604_15750_b200 import DepCap
+    tiny = inputs.scaled(inputs.WORKLOADS["tiny_f32"], n_layers=0, ctx_min=0, ctx_max=0)
+    weights = inputs.make_weights(tiny, device=dev, n_layers=0)
+    eng = DepCap.from_workload(tiny, weights, n_layers=0, max_batch=1, max_window=128, max_ctx=0)
+    B, W = 8192, 128
+    g = torch.Generator(device=dev).manual_seed(1234)
+    rnd = lambda *s: torch.rand(s, device=dev, generator=g)
+    I = (torch.randn((B, W), device=dev, generator=g).abs() * torch.exp(-torch.arange(W, device=dev) / 16.0)).contiguous()
+    H = rnd(B, W) * 8
+    conf = torch.where(rnd(B, W) < 0.5, 0.9 + 0.1 * rnd(B, W), rnd(B, W))
+    x = torch.randn((B, W, W), device=dev, generator=g) * 6 - 12
+    ids = torch.where(rnd(B, W) < 0.8, tiny.mask_id, 5).to(torch.int32)
+    win = torch.full((B,), W, dtype=torch.int32, device=dev)
+    remain = torch.full((B,), 256, dtype=torch.int32, device=dev)
+    bo = dict(score=torch.zeros((B, W), device=dev), cum_influence=torch.zeros((B, W), device=dev),
+              cum_score=torch.zeros((B, W), device=dev), block_len=torch.zeros((B,), dtype=torch.int32, device=dev))
+    so = dict(sel_mask=torch.zeros((B, W), dtype=torch.uint8, device=dev),
+              sel_idx=torch.zeros((B, W), dtype=torch.int32, device=dev),
+              sel_count=torch.zeros((B,), dtype=torch.int32, device=dev))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than L2
+    peaks = _peaks()
+    res = {}
+    # the whole window is the block, so that Algorithm 1 sees pools of about 50 positions; it reads
+    # D_ij only for pairs of pool members (both halves of Eq. 6): bytes touched are counted from
+    # the inputs, the nominal figure is the whole W x W matrix
+    blk = torch.full((B,), W, dtype=torch.int32, device=dev)
+    pool = ((ids == tiny.mask_id) & (conf >= 0.8)).sum(dim=1).double()
+    sel_touched = float((2.0 * pool * (pool - 1) * 4).sum().item()) + B * (W * 4.0 + W * 4 + 8 + W + W * 4 + 4)
+    for name, fn, nbytes, nominal in (
+            ("k_boundary", lambda: eng.boundary_batched(I, H, win, remain, bo), B * (5.0 * W * 4 + 12),
+             B * (5.0 * W * 4 + 12)),
+            ("k_select", lambda: eng.select_batched(conf, ids, x, blk, win, so), sel_touched,
+             B * (W * 4.0 + W * 4 + W * W * 4 + 8 + W + W * 4 + 4))):
+        for _ in range(3):
+            fn()
+        times = []
+        for _ in range(max(5, min(args.steps, 20))):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(eng.stream); fn(); e1.record(eng.stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = float(np.median(times))
+        ach = nbytes / (ms * 1e-3) / 1e9
+        res[name] = dict(ms=ms, algorithmic_bytes=nbytes, nominal_bytes=nominal, achieved=ach, unit="GB/s",
+                         peak=peaks["hbm"], frac=ach / peaks["hbm"], bound="hbm")
+    committed = int(so["sel_count"].sum().item())
+    print(json.dumps(dict(metric="decision_kernels_GBps", mode="decisions", n_gpus=1, sequences=B, window=W,
+                          committed=committed, rooflines=res, peak_source=peaks["source"],
+                          l2="flushed between timed launches (256 MiB fill)", data="synthetic", dtype="f32")),
+          flush=True)
+    eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,12 +391,15 @@ def main():
     ap.add_argument("--no-coop", action="store_true",
                     help="profiling: launch the fused dense kernel without the cooperative attribute "
                          "(ncu cannot replay cooperative cluster launches); same grid, same work")
-    ap.add_argument("--mode", default="step", choices=["step", "generate", "prefill"],
+    ap.add_argument("--mode", default="step", choices=["step", "generate", "prefill", "decisions"],
                     help="step: the bench line; generate / prefill: measurements of the decoding "
                          "loop and of dc_prefill on the same model shape (one GPU, own JSON line)")
     ap.add_argument("--prev", default="recomputed", choices=["recomputed", "carried"],
                     help="step mode: p_prev from a second variant in the pass (the bench line) or from "
                          "rows carried in (DC_STEP_CARRIED_PREV: half the rows through the stack)")
+    ap.add_argument("--ctx", default="prefill", choices=["prefill", "noise"],
+                    help="step mode: the context cache comes from dc_prefill over the seeded prompt "
+                         "(default) or is seeded N(0,1) noise")
     ap.add_argument("--gen-len", type=int, default=256)
     ap.add_argument("--prompt-len", type=int, default=1024)
     ap.add_argument("--lm-scale", type=float, default=8.0,
@@ -351,7 +422,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     if args.mode != "step":
         if rank == 0:
-            (run_generate if args.mode == "generate" else run_prefill)(args, wl, dev)
+            dict(generate=run_generate, prefill=run_prefill, decisions=run_decisions)[args.mode](args, wl, dev)
         return
     dist = None
     if world > 1:
@@ -360,15 +431,28 @@ def main():
     n_layers = args.layers or wl.n_layers
     # each replica draws its own sequences (seed offset by rank); weights are the same model
     wl_r = inputs.scaled(wl, seed=replicas.replica_seed(wl.seed, rank)) if rank else wl
-    weights, k_log, v_log, toks, lens, steer = _setup(wl, dev, n_layers)
+    weights, k_log, v_log, toks, lens, steer = _setup(wl, dev, n_layers, noise_ctx=args.ctx != "prefill")
     if rank:
         toks = inputs.make_tokens(wl_r)
         steer = inputs.make_steering(wl_r, weights["lm_head"], profile="decay")
-    eng = DepCap.from_workload(wl, weights, n_layers=n_layers, impl=1 if args.kernels == "simt" else 0)
+    eng = DepCap.from_workload(wl, weights, n_layers=n_layers, impl=1 if args.kernels == "simt" else 0,
+                               max_last=max(wl.last_len, wl.ctx_max) if args.ctx == "prefill" else None)
     if args.no_coop:
         eng.set_option(1, 0)
     B, W = wl.batch, eng.max_window
-    kc, vc = pack_kv_cache(k_log, v_log, eng.max_batch, eng.max_ctx)
+    if args.ctx == "prefill":
+        # the context cache as the model itself makes it: one bidirectional pass over the prompt
+        kc = torch.zeros((n_layers, eng.max_batch, wl.n_kv_heads, eng.max_ctx, wl.head_dim),
+                         dtype=wl.torch_dtype, device=dev)
+        vc = torch.zeros((n_layers, eng.max_batch, wl.n_kv_heads, wl.head_dim, eng.max_ctx),
+                         dtype=wl.torch_dtype, device=dev)
+        ids = torch.zeros((B, eng.max_last), dtype=torch.int32)
+        ids[:, :wl.ctx_max] = toks["prompt"]
+        eng.prefill(kc, vc, ids.to(dev), lens["ctx_len"])
+        eng.synchronize()
+        assert int(eng.out["status"][:B].abs().max().item()) == 0
+    else:
+        kc, vc = pack_kv_cache(k_log, v_log, eng.max_batch, eng.max_ctx)
     last_h = torch.zeros((B, eng.max_last), dtype=torch.int32).pin_memory()
     last_h[:, :wl.last_len] = toks["last_ids"]
     win_h = torch.full((B, W), wl.mask_id, dtype=torch.int32).pin_memory()
@@ -536,7 +620,8 @@ def main():
     parity = None
     if not args.no_cpu_baseline:
         s = _oracle_sample(inputs.scaled(wl, n_layers=n_layers), weights,
-                           k_log, v_log, toks, lens, steer)
+                           k_log, v_log, toks, lens, steer,
+                           prompt=toks["prompt"] if args.ctx == "prefill" else None)
         dec = []
         oc = _oracle_committed(wl, weights, toks, lens, steer, decisions=dec)
         cpu = dict(value=oc / s["est_step_s"], unit=UNIT, cores=torch.get_num_threads(),
@@ -558,7 +643,8 @@ def main():
                 steps=args.steps, warmup=args.warmup, ms_per_step=ms_step, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16" if wl.dtype == "bf16" else "f32",
                 data="synthetic",
-                config=_config(wl, n_layers, "curr + carried prev rows" if args.prev == "carried" else "curr+prev"),
+                config=_config(wl, n_layers, "curr + carried prev rows" if args.prev == "carried" else "curr+prev",
+                               ctx=args.ctx),
                 committed_per_step=committed, kernels=args.kernels, status=status_bad,
                 clocks=clocks,
                 e2e=dict(value=committed_e2e / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,

@@ -76,13 +76,12 @@ enum {
   DC_STEP_CARRIED_PREV = 8, /* p_prev comes from rows the caller carried over from an earlier step
                             (h_prev_in, prev_len) instead of a second variant in this pass: the
                             stack runs the curr rows only (half the rows).  This is how the
-                            paper's own implementation obtains the two distributions ("logits
-                            immediately before and after decoding B", Implementation
-                            Approximation).  Not together with DC_STEP_INFLUENCE              */
+                            paper's own implementation obtains the two distributions (appendix,
+                            Implementation Approximation).  Not together with DC_STEP_INFLUENCE */
   DC_STEP_EXPORT_KV = 4  /* append the last decoded block's K / V (curr variant, every layer) to
                             the caches at keys ctx_len[b] .. ctx_len[b] + last_len[b] - 1: the
                             library WRITES k_cache / v_cache there (block-wise cache reuse,
-                            Section 4.1 "compatible with existing block-wise cache techniques");
+                            Section 4.1);
                             needs ctx_len[b] + last_len[b] <= max_ctx                        */
 };
 
@@ -111,6 +110,9 @@ typedef struct dc_config {
   int32_t forbid_mask_pred; /* 1: [MASK] is removed from the softmax of both variants       */
   int32_t impl;             /* DC_IMPL_AUTO: tensor-core kernels where the shape allows;     */
                             /* DC_IMPL_SIMT: plain CUDA-core kernels only (any shape)       */
+  int32_t qkv_bias;         /* 1: the q / k / v projections carry biases (dc_weights.bq/bk/bv), */
+                            /* added before the rotation; the Dream backbone (Section 5.1) has */
+                            /* them, LLaDA does not.  0: no biases anywhere                    */
 } dc_config;
 
 /* Borrowed device pointers.  Per-layer members are HOST arrays of n_layers device pointers. */
@@ -127,6 +129,9 @@ typedef struct dc_weights {
   const void* const* norm2;   /* [d_model] gain of the pre-MLP RMSNorm                      */
   const void* final_norm;     /* [d_model]                                                  */
   const void* lm_head;        /* [vocab, d_model] (untied)                                  */
+  const void* const* bq;      /* [n_q_heads*head_dim]   biases of the q / k / v projections; */
+  const void* const* bk;      /* [n_kv_heads*head_dim]  read only when dc_config.qkv_bias,   */
+  const void* const* bv;      /* [n_kv_heads*head_dim]  null otherwise                       */
 } dc_weights;
 
 typedef struct dc_step_in {
@@ -157,6 +162,11 @@ typedef struct dc_step_in {
    * boundary rule ends the block at prev_len[b] at the latest; prev_len[b] = 0 is a cold start. */
   const void* h_prev_in;
   const int32_t* prev_len;
+  /* Optional, host [batch]: absolute position of the first active row (the frontier).  Null: the
+   * rows follow the cached keys, position ctx_len[b] + r.  With a dual cache (the context cache
+   * also holds the masked suffix behind the window, Section 5.2) the number of cached keys is no
+   * longer the frontier's position: pass it here. */
+  const int32_t* pos0;
 } dc_step_in;
 
 /* Caller-owned device buffers; rows b >= batch and columns k >= win_len[b] are not written.
@@ -240,13 +250,24 @@ DC_API int dc_boundary(dc_ctx* ctx, const dc_boundary_in* in, const dc_boundary_
  * previous dc_step wrote (or any caller-made ones). */
 DC_API int dc_select(dc_ctx* ctx, const dc_select_in* in, const dc_select_out* out);
 
-/* ---- the decoding loop around the step (Section 3, Eq. 1-2; Section 4.2 "starting from the
- * current frontier ...") ---------------------------------------------------------------------- */
+/* The two decision kernels over any number of sequences in one call (a serving layer that batches
+ * the decisions of many requests; also what bench.py times for their bandwidth number).  Same
+ * kernels, same arithmetic and layouts as dc_boundary / dc_select (row pitch max_window of the
+ * context), but the per-sequence lengths are DEVICE arrays [batch] and batch is not limited by
+ * max_batch.  have_prev may be null (= all 1).  Section 4.2 / 4.4 and Algorithm 1. */
+DC_API int dc_boundary_batched(dc_ctx* ctx, int32_t batch, const float* influence, const float* entropy,
+                               const int32_t* win_len, const int32_t* remain_len, const int32_t* have_prev,
+                               const dc_boundary_out* out);
+DC_API int dc_select_batched(dc_ctx* ctx, int32_t batch, const float* conf, const int32_t* win_ids,
+                             const float* xlogp, const int32_t* block_len, const int32_t* win_len,
+                             const dc_select_out* out);
+
+/* ---- the decoding loop around the step (Section 3, Eq. 1-2; forward scan of Section 4.2) ----- */
 
 /* Prefill: the K / V of n_ids[b] clean tokens per sequence (a prompt, or any run of decoded
  * tokens whose cache is to be rebuilt), computed by one bidirectional pass over those tokens - they
  * attend one another and the ctx_len[b] keys already in the cache (Section 3: the DLM attends the
- * whole known sequence; Section 4.1 / "compatible with existing block-wise cache techniques") -
+ * whole known sequence; block-wise cache reuse, Section 4.1) -
  * and written into the caches at keys ctx_len[b] .. ctx_len[b] + n_ids[b] - 1, every layer.  The
  * same kernels as dc_step without window rows; no LM head.  A prompt goes through in one call
  * (the pass is bidirectional, so chunks would not see each other): n_ids[b] <= max_last and
@@ -258,6 +279,12 @@ typedef struct dc_prefill_in {
   const int32_t* ctx_len;    /* host [batch], may be null (all 0)                             */
   const int32_t* ids;        /* device [batch][max_last]                                      */
   const int32_t* n_ids;      /* host [batch]                                                  */
+  const int32_t* pos0;       /* host [batch] or null: absolute position of ids[b][0]; null means
+                                ctx_len[b] (the tokens follow the cached ones).  Other values are
+                                for cached rows that do not follow the context in the sequence -
+                                the still masked suffix behind the window that a dual cache keeps
+                                (Section 5.2, cache compatibility): K is stored rotated, so the
+                                position is all a later step needs to know about such a row      */
 } dc_prefill_in;
 typedef struct dc_prefill_out {
   int32_t* status;           /* device [batch]                                                */
@@ -318,8 +345,15 @@ DC_API int dc_generate(dc_ctx* ctx, const dc_generate_in* in, const dc_generate_
  *     that cannot replay cooperative cluster launches.  All CTAs are still resident when the GPU
  *     runs nothing else, and every wait in the kernel is bounded (DC_ERR_TIMEOUT in status[b]
  *     otherwise), but the guarantee is gone: not for production use.
- * Returns DC_ERR_INVALID_ARG for an unknown option. */
-enum { DC_OPT_COOPERATIVE = 1 };
+ *   DC_OPT_WAIT_LIMIT_US (default 2 000 000): how long a device-side wait (on a TMA / MMA
+ *     barrier, the grid barrier, a hand-over flag) polls before the kernel gives up, frees what it
+ *     holds, returns and reports DC_ERR_TIMEOUT in status[b]; 1000 .. 60 000 000.  The value is
+ *     kept on the device and is shared by every context of the process on that device.
+ *   DC_OPT_TEST_STALL_LMHEAD (default 0): test hook for the path above.  1 makes the LM-head
+ *     kernel skip all of its loads, so that nothing is in flight and every one of its waits runs
+ *     out: the step then ends with DC_ERR_TIMEOUT in every status[b] and the context stays usable.
+ * Returns DC_ERR_INVALID_ARG for an unknown option or a value out of range. */
+enum { DC_OPT_COOPERATIVE = 1, DC_OPT_WAIT_LIMIT_US = 2, DC_OPT_TEST_STALL_LMHEAD = 3 };
 DC_API int dc_set_option(dc_ctx* ctx, int32_t option, int32_t value);
 
 /* Frees the workspace.  The caller must have synchronised the stream.  Null is a no-op. */

@@ -219,16 +219,19 @@ def forward(cfg: OracleConfig, w: OracleWeights, tok: np.ndarray, pos0: int,
 
 
 def prefill(cfg: OracleConfig, w: OracleWeights, ids: np.ndarray, k_ctx=None, v_ctx=None,
-            ctx_len: int = 0, n_layers: int | None = None):
+            ctx_len: int = 0, n_layers: int | None = None, pos0: int | None = None):
     """K / V of a run of clean tokens (a prompt), as one bidirectional pass over them makes
     them: the tokens sit at positions ctx_len + r, attend one another and the ctx_len cached
     keys (Section 3: the model attends the whole known sequence, no causal mask).
+    pos0: position of ids[0] when the tokens do not follow the cached ones in the sequence (the
+    still masked suffix behind the window that a dual cache keeps, Section 5.2): attention is
+    bidirectional and K carries its rotation, so a cached row's position matters only here.
     Returns (k, v), each [n_layers, n_kv_heads, len(ids), head_dim], K rotated.
     """
     if k_ctx is not None:
         k_ctx, v_ctx = k_ctx[:, :, :ctx_len, :], v_ctx[:, :, :ctx_len, :]
-    _, kv = forward(cfg, w, np.asarray(ids), int(ctx_len), k_ctx, v_ctx, return_kv=True,
-                    n_layers=n_layers)
+    _, kv = forward(cfg, w, np.asarray(ids), int(ctx_len if pos0 is None else pos0), k_ctx, v_ctx,
+                    return_kv=True, n_layers=n_layers)
     k = np.stack([np.transpose(k_, (1, 0, 2)) for k_, _ in kv])
     v = np.stack([np.transpose(v_, (1, 0, 2)) for _, v_ in kv])
     return k, v
@@ -407,14 +410,17 @@ def cap_select(conf: np.ndarray, masked: np.ndarray, xlogp: np.ndarray, block_le
 def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
          last_ids: np.ndarray, win_ids: np.ndarray, remain_len: int,
          influence: bool = True, h_final=None, n_layers: int | None = None,
-         return_kv: bool = False, carried=None) -> dict:
+         return_kv: bool = False, carried=None, pos0: int | None = None) -> dict:
     """All per-step outputs for one sequence.
 
     curr variant rows = last decoded block followed by the window; prev variant = the same
     rows with the last block's ids replaced by [MASK] (everything else fixed), so that
     p_prev = p(Z_k | c) and p_curr = p(Z_k | c, b).  h_final, if given, is
     (h_curr [W,d], h_prev [W,d] or None) and replaces the transformer stack's output.
+    pos0: position of the first active row; default ctx_len (the rows follow the cached keys).
+    With a dual cache the context also holds suffix rows, and the frontier's position is given.
     """
+    pos0 = int(ctx_len if pos0 is None else pos0)
     Lb, W = len(last_ids), len(win_ids)
     have_prev = bool(influence and Lb > 0)
     if carried is not None:
@@ -428,7 +434,7 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
         k_ctx, v_ctx = k_ctx[:, :, :ctx_len, :], v_ctx[:, :, :ctx_len, :]
     if h_final is None:
         tok_curr = np.concatenate([last_ids, win_ids]).astype(np.int64)
-        x = forward(cfg, w, tok_curr, ctx_len, k_ctx, v_ctx, n_layers=n_layers,
+        x = forward(cfg, w, tok_curr, pos0, k_ctx, v_ctx, n_layers=n_layers,
                     return_kv=return_kv)
         kv_last = None
         if return_kv:  # K / V of the last decoded block's rows, as this (curr) forward made them
@@ -439,7 +445,7 @@ def step(cfg: OracleConfig, w: OracleWeights, k_ctx, v_ctx, ctx_len: int,
         if have_prev:
             tok_prev = tok_curr.copy()
             tok_prev[:Lb] = cfg.mask_id
-            xp = forward(cfg, w, tok_prev, ctx_len, k_ctx, v_ctx, n_layers=n_layers)
+            xp = forward(cfg, w, tok_prev, pos0, k_ctx, v_ctx, n_layers=n_layers)
             h_prev = final_hidden(cfg, w, xp[Lb:])
     else:
         kv_last = None

@@ -21,8 +21,8 @@ STAGE_NAMES = ["embed", "norm", "qkv", "attn", "oproj", "gateup", "down", "lmhea
                "boundary", "dense"]
 EXPORTS = ["dc_create", "dc_step", "dc_boundary", "dc_select", "dc_destroy", "dc_last_error",
            "dc_debug_logits", "dc_step_profiled", "dc_signals_static", "dc_commit", "dc_generate", "dc_prefill",
-           "dc_set_option"]
-DC_OPT_COOPERATIVE = 1
+           "dc_set_option", "dc_boundary_batched", "dc_select_batched"]
+DC_OPT_COOPERATIVE, DC_OPT_WAIT_LIMIT_US, DC_OPT_TEST_STALL_LMHEAD = 1, 2, 3
 
 
 class DepCapError(RuntimeError):
@@ -40,7 +40,7 @@ class dc_config(C.Structure):
                [("lambda_", C.c_float), ("L_min", C.c_int32), ("L_max", C.c_int32),
                 ("tau_low", C.c_float), ("tau_high", C.c_float), ("gamma", C.c_float)] + \
                [(n, C.c_int32) for n in ("smooth_radius", "norm_mode", "boundary_mode",
-                                         "cap_mode", "forbid_mask_pred", "impl")]
+                                         "cap_mode", "forbid_mask_pred", "impl", "qkv_bias")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -50,7 +50,8 @@ class dc_weights(C.Structure):
     _fields_ = [("embed", C.c_void_p)] + \
                [(n, _PP) for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm1",
                                    "norm2")] + \
-               [("final_norm", C.c_void_p), ("lm_head", C.c_void_p)]
+               [("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + \
+               [(n, _PP) for n in ("bq", "bk", "bv")]
 
 
 _I32P = C.POINTER(C.c_int32)
@@ -61,7 +62,7 @@ class dc_step_in(C.Structure):
                 ("v_cache", C.c_void_p), ("ctx_len", _I32P), ("last_ids", C.c_void_p),
                 ("last_len", _I32P), ("win_ids", C.c_void_p), ("win_len", _I32P),
                 ("remain_len", _I32P), ("h_final_in", C.c_void_p), ("h_prev_in", C.c_void_p),
-                ("prev_len", _I32P)]
+                ("prev_len", _I32P), ("pos0", _I32P)]
 
 
 class dc_step_out(C.Structure):
@@ -92,7 +93,7 @@ class dc_select_out(C.Structure):
 
 class dc_prefill_in(C.Structure):
     _fields_ = [("batch", C.c_int32), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
-                ("ctx_len", _I32P), ("ids", C.c_void_p), ("n_ids", _I32P)]
+                ("ctx_len", _I32P), ("ids", C.c_void_p), ("n_ids", _I32P), ("pos0", _I32P)]
 
 
 class dc_prefill_out(C.Structure):
@@ -158,6 +159,8 @@ def load_library(path: str | None = None):
     lib_.dc_generate.argtypes = [C.c_void_p, C.POINTER(dc_generate_in),
                                  C.POINTER(dc_generate_out)]
     lib_.dc_destroy.argtypes = [C.c_void_p]
+    lib_.dc_boundary_batched.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 5 + [C.POINTER(dc_boundary_out)]
+    lib_.dc_select_batched.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 5 + [C.POINTER(dc_select_out)]
     lib_.dc_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib_.dc_debug_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
     lib_.dc_last_error.argtypes = [C.c_void_p]
@@ -263,7 +266,8 @@ class DepCap:
                         tau_low=hyper.tau_low, tau_high=hyper.tau_high, gamma=hyper.gamma,
                         smooth_radius=hyper.smooth_radius, norm_mode=hyper.norm_mode,
                         boundary_mode=hyper.boundary_mode, cap_mode=hyper.cap_mode,
-                        forbid_mask_pred=int(hyper.forbid_mask_pred), impl=impl)
+                        forbid_mask_pred=int(hyper.forbid_mask_pred), impl=impl,
+                        qkv_bias=int(n_layers > 0 and "bq" in weights["layers"][0]))
         self._weights = weights          # keep the borrowed tensors alive
         layers = weights["layers"][:n_layers]
         for t in [weights["embed"], weights["lm_head"], weights["final_norm"]] + \
@@ -276,6 +280,11 @@ class DepCap:
             arr = (C.c_void_p * max(n_layers, 1))(*[lw[name].data_ptr() for lw in layers])
             self._arrays.append(arr)
             setattr(w, name, C.cast(arr, _PP))
+        if cfg.qkv_bias:     # the layers carry biases of the q / k / v projections ("bq", "bk", "bv")
+            for name in ("bq", "bk", "bv"):
+                arr = (C.c_void_p * n_layers)(*[lw[name].data_ptr() for lw in layers])
+                self._arrays.append(arr)
+                setattr(w, name, C.cast(arr, _PP))
         with torch.cuda.device(self.device):
             rc = self._lib.dc_create(C.byref(cfg), C.byref(w), C.c_void_p(self.stream.cuda_stream),
                                      C.byref(self._ctx))
@@ -313,7 +322,7 @@ class DepCap:
     # -- dc_step ---------------------------------------------------------------------------
     def _step_structs(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len,
                       remain_len, influence=True, boundary=True, h_final=None, want_xlogp=True,
-                      export_kv=False, carried=None, h_out=None):
+                      export_kv=False, carried=None, h_out=None, pos0=None):
         B = len(win_len)
         self._keep = (k_cache, v_cache, last_ids, win_ids, h_final,
                       _host_i32(ctx_len, B), _host_i32(last_len, B), _host_i32(win_len, B),
@@ -333,6 +342,9 @@ class DepCap:
         if carried is not None:
             si.h_prev_in = _ptr(self._keep_c[0])
             si.prev_len = C.cast(self._keep_c[1], _I32P)
+        if pos0 is not None:
+            self._keep_p0 = _host_i32(pos0, B)
+            si.pos0 = C.cast(self._keep_p0, _I32P)
         so = dc_step_out(**{k: _ptr(v) for k, v in self.out.items()})
         if not want_xlogp:
             so.xlogp = None
@@ -342,13 +354,13 @@ class DepCap:
 
     def step(self, k_cache, v_cache, ctx_len, last_ids, last_len, win_ids, win_len, remain_len,
              influence=True, boundary=True, h_final=None, export_kv=False, carried=None,
-             h_out=None, want_xlogp=True):
+             h_out=None, want_xlogp=True, pos0=None):
         """Enqueue one block-step (dc_step).  Device tensors in, self.out (device) filled.
         export_kv: also append the last block's K / V to the caches (which are then written)."""
         si, so = self._step_structs(k_cache, v_cache, ctx_len, last_ids, last_len, win_ids,
                                     win_len, remain_len, influence, boundary, h_final,
                                     want_xlogp=want_xlogp, export_kv=export_kv, carried=carried,
-                                    h_out=h_out)
+                                    h_out=h_out, pos0=pos0)
         self._check(self._lib.dc_step(self._ctx, C.byref(si), C.byref(so)))
         return self.out
 
@@ -392,15 +404,37 @@ class DepCap:
         self._check(self._lib.dc_select(self._ctx, C.byref(si), C.byref(so)))
         return self.sel
 
-    def prefill(self, k_cache, v_cache, ids, n_ids, ctx_len=None):
+    def boundary_batched(self, influence, entropy, win_len, remain_len, out, have_prev=None):
+        """dc_boundary_batched: device length arrays, any batch; `out` maps score / cum_influence /
+        cum_score / block_len to device tensors ([batch, max_window]; block_len [batch])."""
+        bo = dc_boundary_out(**{k: _ptr(out.get(k)) for k in ("score", "cum_influence", "cum_score",
+                                                              "block_len")})
+        self._check(self._lib.dc_boundary_batched(self._ctx, influence.shape[0], _ptr(influence),
+                                                  _ptr(entropy), _ptr(win_len), _ptr(remain_len),
+                                                  _ptr(have_prev), C.byref(bo)))
+        return out
+
+    def select_batched(self, conf, win_ids, xlogp, block_len, win_len, out):
+        """dc_select_batched: device length array, any batch; `out` maps sel_mask / sel_idx /
+        sel_count to device tensors."""
+        so = dc_select_out(**{k: _ptr(out.get(k)) for k in ("sel_mask", "sel_idx", "sel_count")})
+        self._check(self._lib.dc_select_batched(self._ctx, conf.shape[0], _ptr(conf), _ptr(win_ids),
+                                                _ptr(xlogp), _ptr(block_len), _ptr(win_len),
+                                                C.byref(so)))
+        return out
+
+    def prefill(self, k_cache, v_cache, ids, n_ids, ctx_len=None, pos0=None):
         """K / V of n_ids[b] clean tokens (device ids [B, max_last]) into the caches at keys
-        ctx_len[b] ...; returns the device status tensor."""
+        ctx_len[b] ...; pos0: the tokens' absolute positions when they are not ctx_len[b] ...;
+        returns the device status tensor."""
         B = len(n_ids)
         n_ = _host_i32(n_ids, B)
         c_ = _host_i32(ctx_len if ctx_len is not None else [0] * B, B)
-        self._keep_pf = (k_cache, v_cache, ids, n_, c_)
+        p_ = _host_i32(pos0, B) if pos0 is not None else None
+        self._keep_pf = (k_cache, v_cache, ids, n_, c_, p_)
         pi = dc_prefill_in(batch=B, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
-                           ctx_len=C.cast(c_, _I32P), ids=_ptr(ids), n_ids=C.cast(n_, _I32P))
+                           ctx_len=C.cast(c_, _I32P), ids=_ptr(ids), n_ids=C.cast(n_, _I32P),
+                           pos0=C.cast(p_, _I32P) if p_ is not None else None)
         po = dc_prefill_out(status=_ptr(self.out["status"]))
         self._check(self._lib.dc_prefill(self._ctx, C.byref(pi), C.byref(po)))
         return self.out["status"]

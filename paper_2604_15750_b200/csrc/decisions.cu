@@ -65,18 +65,25 @@ __device__ __forceinline__ float normalise(float x, float hi, float lo, int mode
   return __fdiv_rn(__fsub_rn(x, lo), fmaxf(__fsub_rn(hi, lo), 1e-8f));
 }
 
+// Lengths of the sequences of a call: by value inside SeqMeta (a step: at most DC_MAX_BATCH
+// sequences), or - when the pointers are set - arrays in device memory, for calls over any number
+// of sequences.
+__device__ __forceinline__ int len_of(const int32_t* dev, const int* by_value, int b) {
+  return dev != nullptr ? dev[b] : by_value[b];
+}
+
 __global__ void __launch_bounds__(kThreads) k_boundary(
     const float* __restrict__ influence, const float* __restrict__ entropy, int ld, SeqMeta m,
-    Hyper hp, int max_window, float* __restrict__ score, float* __restrict__ cum_i,
+    DevLens dl, Hyper hp, int max_window, float* __restrict__ score, float* __restrict__ cum_i,
     float* __restrict__ cum_s, int32_t* __restrict__ block_len) {
   __shared__ float sI[kMaxW], sH[kMaxW];
   __shared__ float redf[kThreads / 32];
   __shared__ int redi[kThreads / 32];
   __shared__ long long wtot[kThreads / 32];
   const int b = blockIdx.x, k = threadIdx.x;
-  const int Lw = max(0, min(min(hp.L_max, m.remain[b]), m.win_len[b]));
+  const int Lw = max(0, min(min(hp.L_max, len_of(dl.remain, m.remain, b)), len_of(dl.win_len, m.win_len, b)));
   const size_t o = (size_t)b * max_window + k;
-  if (!m.have_prev[b]) {  // cold start: the first block uses L_min
+  if (!len_of(dl.have_prev, m.have_prev, b)) {  // cold start: the first block uses L_min
     if (k < Lw) {
       if (score) score[o] = 0.f;
       if (cum_i) cum_i[o] = 0.f;
@@ -121,8 +128,15 @@ __global__ void __launch_bounds__(kThreads) k_boundary(
 void launch_boundary(const float* influence, const float* entropy, int ld, const SeqMeta& m,
                      const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
                      int32_t* block_len, cudaStream_t s) {
-  k_boundary<<<m.batch, kThreads, 0, s>>>(influence, entropy, ld, m, hp, max_window, score, cum_i,
-                                          cum_s, block_len);
+  k_boundary<<<m.batch, kThreads, 0, s>>>(influence, entropy, ld, m, DevLens{}, hp, max_window, score,
+                                          cum_i, cum_s, block_len);
+}
+
+void launch_boundary_dev(const float* influence, const float* entropy, int ld, int batch, const DevLens& dl,
+                         const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
+                         int32_t* block_len, cudaStream_t s) {
+  k_boundary<<<batch, kThreads, 0, s>>>(influence, entropy, ld, SeqMeta{}, dl, hp, max_window, score,
+                                        cum_i, cum_s, block_len);
 }
 
 // ---- CAP-Decoding ------------------------------------------------------------------------------
@@ -154,9 +168,9 @@ __device__ void greedy_pass(const uint32_t* cand, const int* order, int n_order,
 
 __global__ void __launch_bounds__(kThreads) k_select(
     const float* __restrict__ conf, const int32_t* __restrict__ win_ids,
-    const float* __restrict__ xlogp, const int32_t* __restrict__ block_len, SeqMeta m, Hyper hp,
-    int mask_id, int max_window, uint8_t* __restrict__ sel_mask, int32_t* __restrict__ sel_idx,
-    int32_t* __restrict__ sel_count) {
+    const float* __restrict__ xlogp, const int32_t* __restrict__ block_len, SeqMeta m, DevLens dl,
+    Hyper hp, int mask_id, int max_window, uint8_t* __restrict__ sel_mask,
+    int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_count) {
   __shared__ float sc[kMaxW];
   __shared__ uint32_t s_block[kWords], s_pool[kWords], s_hi[kWords], s_sel[kWords],
       s_cand[kWords], s_alive[kWords];
@@ -164,7 +178,7 @@ __global__ void __launch_bounds__(kThreads) k_select(
   __shared__ int s_order[kMaxW];
   __shared__ int s_n;
   const int b = blockIdx.x, i = threadIdx.x;
-  const int W = m.win_len[b];
+  const int W = len_of(dl.win_len, m.win_len, b);
   const int L = min(max(block_len[b], 0), W);
   const bool in_block = i < L && win_ids[(size_t)b * max_window + i] == mask_id;  // M^t ∩ B^t
   const float c = (i < W) ? conf[(size_t)b * max_window + i] : 0.f;
@@ -272,8 +286,16 @@ void launch_select(const float* conf, const int32_t* win_ids, const float* xlogp
                    const int32_t* block_len, const SeqMeta& m, const Hyper& hp, int mask_id,
                    int max_window, uint8_t* sel_mask, int32_t* sel_idx, int32_t* sel_count,
                    cudaStream_t s) {
-  k_select<<<m.batch, kThreads, 0, s>>>(conf, win_ids, xlogp, block_len, m, hp, mask_id,
+  k_select<<<m.batch, kThreads, 0, s>>>(conf, win_ids, xlogp, block_len, m, DevLens{}, hp, mask_id,
                                         max_window, sel_mask, sel_idx, sel_count);
+}
+
+void launch_select_dev(const float* conf, const int32_t* win_ids, const float* xlogp,
+                       const int32_t* block_len, int batch, const DevLens& dl, const Hyper& hp, int mask_id,
+                       int max_window, uint8_t* sel_mask, int32_t* sel_idx, int32_t* sel_count,
+                       cudaStream_t s) {
+  k_select<<<batch, kThreads, 0, s>>>(conf, win_ids, xlogp, block_len, SeqMeta{}, dl, hp, mask_id,
+                                      max_window, sel_mask, sel_idx, sel_count);
 }
 
 // ---- commit (Eq. 2): y_i <- yhat_i for the selected positions; masked positions left in the block --

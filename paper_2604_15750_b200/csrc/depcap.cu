@@ -67,6 +67,7 @@ struct dc_ctx {
   bool tc_lm = false;   // tensor-core LM head fused with the streaming softmax statistics
   const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
   std::vector<const void*> wq, wk, wv, wo, w_gate, w_up, w_down, norm1, norm2;
+  std::vector<const void*> bq, bk, bv;   // q / k / v projection biases (cfg.qkv_bias), else empty
   // capacities
   int R_cap_max = 0, M_max = 0, Mlm_max = 0;
   // workspace (device)
@@ -145,6 +146,7 @@ int build_meta(dc_ctx* c, int batch, int flags, const int32_t* ctx_len, const in
       return fail(c, DC_ERR_SHAPE, "win_len[%d]=%d outside [1, max_window=%d]", b, W,
                   g.max_window);
     m->ctx_len[b] = P; m->last_len[b] = Lb; m->win_len[b] = W;
+    m->pos0[b] = P;   // active rows sit right behind the cached context
     m->remain[b] = remain_len ? remain_len[b] : W;
     m->have_prev[b] = (m->nv == 2 && Lb > 0) ? 1 : 0;
     maxR = maxR > Lb + W ? maxR : Lb + W;
@@ -263,7 +265,9 @@ int run_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, const SeqM
                         EPI_STORE_F32, s);
     launch_gemm_simt<T>(a, (const T*)c->wv[l], c->tmp + (nq + nkv) * hd, M, nkv * hd, d, nqkv,
                         EPI_STORE_F32, s);
-    launch_rope_store<T>(c->tmp, c->cos_sin, m, nq, nkv, hd, q, k, v, s);
+    launch_rope_store<T>(c->tmp, c->cos_sin, m, nq, nkv, hd,
+                         c->bq.empty() ? nullptr : (const T*)c->bq[l], c->bq.empty() ? nullptr : (const T*)c->bk[l],
+                         c->bq.empty() ? nullptr : (const T*)c->bv[l], q, k, v, s);
     pf.end();
     if (export_kv)
       launch_export_kv<T>(k, v, 0, m, nkv, hd, g.max_ctx, (T*)in->k_cache + (size_t)l * k_layer,
@@ -361,6 +365,11 @@ int validate_step(dc_ctx* c, const dc_step_in* in, const dc_step_out* out, SeqMe
   int rc = build_meta(c, in->batch, in->flags, in->ctx_len, in->last_len, in->win_len,
                       in->remain_len, m);
   if (rc != DC_OK) return rc;
+  if (in->pos0)
+    for (int b = 0; b < m->batch; ++b) {
+      if (in->pos0[b] < 0) return fail(c, DC_ERR_INVALID_ARG, "pos0[%d] negative", b);
+      m->pos0[b] = in->pos0[b];
+    }
   bool any_ctx = false, any_last = false;
   for (int b = 0; b < m->batch; ++b) {
     any_ctx |= m->ctx_len[b] > 0;
@@ -446,6 +455,13 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
   if (g.n_layers > 0 && (!w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
                          !w->w_down || !w->norm1 || !w->norm2))
     return fail(nullptr, DC_ERR_INVALID_ARG, "null per-layer weight array");
+  if (g.qkv_bias != 0 && g.qkv_bias != 1) return fail(nullptr, DC_ERR_INVALID_ARG, "qkv_bias must be 0 or 1");
+  if (g.qkv_bias && g.n_layers > 0) {
+    if (!w->bq || !w->bk || !w->bv) return fail(nullptr, DC_ERR_INVALID_ARG, "qkv_bias set but bq / bk / bv null");
+    for (int l = 0; l < g.n_layers; ++l)
+      if (!w->bq[l] || !w->bk[l] || !w->bv[l])
+        return fail(nullptr, DC_ERR_INVALID_ARG, "null bias pointer in layer %d", l);
+  }
   for (int l = 0; l < g.n_layers; ++l)
     if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] ||
         !w->w_down[l] || !w->norm1[l] || !w->norm2[l])
@@ -470,6 +486,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
     cp(c->wq, w->wq); cp(c->wk, w->wk); cp(c->wv, w->wv); cp(c->wo, w->wo);
     cp(c->w_gate, w->w_gate); cp(c->w_up, w->w_up); cp(c->w_down, w->w_down);
     cp(c->norm1, w->norm1); cp(c->norm2, w->norm2);
+    if (g.qkv_bias) { cp(c->bq, w->bq); cp(c->bk, w->bk); cp(c->bv, w->bv); }
   }
   c->use_tc = g.impl == DC_IMPL_AUTO && tc_supported(g);
   c->tc_lm = c->use_tc && tc_has_lmhead(g);
@@ -516,6 +533,7 @@ int dc_create(const dc_config* cfg, const dc_weights* w, void* cuda_stream, dc_c
       dc_destroy(c);
       return fail(nullptr, rc, "%s", why.c_str());
     }
+    if (g.qkv_bias) tc_set_qkv_bias(c->tc, c->bq, c->bk, c->bv);
   } else {
     c->q = ws_alloc<char>(c, M * nq * hd * es, &ok);
     c->k = ws_alloc<char>(c, M * nkv * hd * es, &ok);
@@ -579,6 +597,39 @@ int dc_select(dc_ctx* c, const dc_select_in* in, const dc_select_out* out) {
   return DC_OK;
 }
 
+int dc_boundary_batched(dc_ctx* c, int32_t batch, const float* influence, const float* entropy,
+                        const int32_t* win_len, const int32_t* remain_len, const int32_t* have_prev,
+                        const dc_boundary_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!influence || !entropy || !win_len || !remain_len || !out || !out->block_len || batch < 1)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument or batch < 1");
+  DevLens dl;
+  dl.win_len = win_len; dl.remain = remain_len; dl.have_prev = have_prev;
+  if (!have_prev) {   // all 1: any non-zero array of the right length serves; win_len >= 1 everywhere
+    dl.have_prev = win_len;
+  }
+  launch_boundary_dev(influence, entropy, c->cfg.max_window, batch, dl, c->hp, c->cfg.max_window,
+                      out->score, out->cum_influence, out->cum_score, out->block_len, c->stream);
+  DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
+int dc_select_batched(dc_ctx* c, int32_t batch, const float* conf, const int32_t* win_ids,
+                      const float* xlogp, const int32_t* block_len, const int32_t* win_len,
+                      const dc_select_out* out) {
+  if (!c) return DC_ERR_INVALID_ARG;
+  if (!conf || !win_ids || !xlogp || !block_len || !win_len || !out || batch < 1)
+    return fail(c, DC_ERR_INVALID_ARG, "null argument or batch < 1");
+  if (!out->sel_mask && !out->sel_idx && !out->sel_count)
+    return fail(c, DC_ERR_INVALID_ARG, "no output requested");
+  DevLens dl;
+  dl.win_len = win_len;
+  launch_select_dev(conf, win_ids, xlogp, block_len, batch, dl, c->hp, c->cfg.mask_id, c->cfg.max_window,
+                    out->sel_mask, out->sel_idx, out->sel_count, c->stream);
+  DC_CHECK_LAUNCH(c);
+  return DC_OK;
+}
+
 int dc_prefill(dc_ctx* c, const dc_prefill_in* in, const dc_prefill_out* out) {
   if (!c) return DC_ERR_INVALID_ARG;
   if (!in || !out || !in->ids || !in->n_ids || !in->k_cache || !in->v_cache || !out->status)
@@ -592,6 +643,11 @@ int dc_prefill(dc_ctx* c, const dc_prefill_in* in, const dc_prefill_out* out) {
       return fail(c, DC_ERR_SHAPE, "ctx_len[%d] + n_ids[%d] = %d exceeds max_ctx=%d", b, b,
                   m.ctx_len[b] + m.last_len[b], c->cfg.max_ctx);
   }
+  if (in->pos0)   // the tokens' positions are not the cache slots (suffix rows of a dual cache)
+    for (int b = 0; b < m.batch; ++b) {
+      if (in->pos0[b] < 0) return fail(c, DC_ERR_INVALID_ARG, "pos0[%d] negative", b);
+      m.pos0[b] = in->pos0[b];
+    }
   dc_step_in si{};
   si.batch = in->batch; si.flags = DC_STEP_EXPORT_KV;
   si.k_cache = in->k_cache; si.v_cache = in->v_cache; si.ctx_len = in->ctx_len;
@@ -760,6 +816,16 @@ int dc_set_option(dc_ctx* c, int32_t option, int32_t value) {
   if (!c) return DC_ERR_INVALID_ARG;
   if (option == DC_OPT_COOPERATIVE) {
     if (c->tc) tc_set_cooperative(c->tc, value != 0);
+    return DC_OK;
+  }
+  if (option == DC_OPT_WAIT_LIMIT_US) {
+    if (value < 1000 || value > 60000000) return fail(c, DC_ERR_INVALID_ARG, "wait limit outside [1000, 60000000] us");
+    if (!c->tc) return DC_OK;   // the CUDA-core kernels have no device-side waits
+    const int rc = tc_set_wait_limit_us(c->tc, value);
+    return rc == DC_OK ? DC_OK : fail(c, rc, "%s", tc_error(c->tc));
+  }
+  if (option == DC_OPT_TEST_STALL_LMHEAD) {
+    if (c->tc) tc_set_stall_lmhead(c->tc, value != 0);
     return DC_OK;
   }
   return fail(c, DC_ERR_INVALID_ARG, "unknown option %d", option);

@@ -18,6 +18,7 @@ struct SeqMeta {
   int win_len[DC_MAX_BATCH];
   int remain[DC_MAX_BATCH];
   int have_prev[DC_MAX_BATCH];
+  int pos0[DC_MAX_BATCH];   // absolute position of active row 0 (ctx_len unless a prefill says otherwise)
   int batch;     // B
   int nv;        // variants in the pass: 1 (curr) or 2 (curr, prev)
   int R_cap;     // active rows per (variant, sequence), multiple of 16: [last ; window ; pad]
@@ -79,10 +80,11 @@ void launch_gemm_simt(const T* A, const T* W, float* C, int M, int N, int K, int
 void launch_rope_table(const SeqMeta& m, int head_dim, float theta, float* cos_sin,
                        cudaStream_t s);
 
-// q,k: rotate + store as T; v: store as T.  tmp layout [M, (nq + 2 nkv) * hd] fp32.
+// q,k: (+ bias) rotate + store as T; v: (+ bias) store as T.  tmp layout [M, (nq + 2 nkv) * hd]
+// fp32; bq / bk / bv: projection biases or null.
 template <typename T>
 void launch_rope_store(const float* tmp, const float* cos_sin, const SeqMeta& m, int nq, int nkv,
-                       int hd, T* q, T* k, T* v, cudaStream_t s);
+                       int hd, const T* bq, const T* bk, const T* bv, T* q, T* k, T* v, cudaStream_t s);
 
 template <typename T>
 void launch_swiglu(const float* gate_up, int M, int F, T* act, cudaStream_t s);
@@ -116,10 +118,25 @@ void launch_export_kv(const T* k, const T* v, int v_ld, const SeqMeta& m, int nk
                       int max_ctx, T* k_cache, T* v_cache, cudaStream_t s);
 
 // ---- decision kernels --------------------------------------------------------------------------
+// per-sequence lengths in device memory (all null: the lengths inside SeqMeta are used)
+struct DevLens {
+  const int32_t* win_len = nullptr;
+  const int32_t* remain = nullptr;
+  const int32_t* have_prev = nullptr;
+};
 // influence/entropy rows have stride `ld`; outputs have stride max_window.
 void launch_boundary(const float* influence, const float* entropy, int ld, const SeqMeta& m,
                      const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
                      int32_t* block_len, cudaStream_t s);
+
+// the same kernel over `batch` sequences (any number) whose lengths are arrays in device memory
+void launch_boundary_dev(const float* influence, const float* entropy, int ld, int batch, const DevLens& dl,
+                         const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
+                         int32_t* block_len, cudaStream_t s);
+void launch_select_dev(const float* conf, const int32_t* win_ids, const float* xlogp,
+                       const int32_t* block_len, int batch, const DevLens& dl, const Hyper& hp, int mask_id,
+                       int max_window, uint8_t* sel_mask, int32_t* sel_idx, int32_t* sel_count,
+                       cudaStream_t s);
 
 void launch_select(const float* conf, const int32_t* win_ids, const float* xlogp,
                    const int32_t* block_len, const SeqMeta& m, const Hyper& hp, int mask_id,

@@ -299,7 +299,7 @@ void launch_gemm_simt(const T* A, const T* W, float* C, int M, int N, int K, int
 
 // ---- RoPE ----------------------------------------------------------------------------------------
 // cos_sin[(b * R_cap + r) * hd + i] = cos(angle), [.. + hd/2 + i] = sin(angle),
-// angle = (ctx_len[b] + r) * theta^(-2i/hd), evaluated in double precision.  Row batch * R_cap
+// angle = (pos0[b] + r) * theta^(-2i/hd), evaluated in double precision.  Row batch * R_cap
 // holds cos / sin of theta^(-2i/hd) itself, the angle step between consecutive rows.
 __global__ void k_rope_table(SeqMeta m, int hd, float theta, float* __restrict__ cos_sin) {
   const int half = hd / 2;
@@ -310,7 +310,7 @@ __global__ void k_rope_table(SeqMeta m, int hd, float theta, float* __restrict__
   const int i = idx % half, br = idx / half;
   const int r = br % m.R_cap, b = br / m.R_cap;
   const double inv_freq = pow((double)theta, -2.0 * (double)i / (double)hd);
-  const double ang = (br < rows) ? (double)(m.ctx_len[b] + r) * inv_freq : inv_freq;
+  const double ang = (br < rows) ? (double)(m.pos0[b] + r) * inv_freq : inv_freq;
   double sn, cs;
   sincos(ang, &sn, &cs);
   cos_sin[(size_t)br * hd + i] = (float)cs;
@@ -325,7 +325,8 @@ void launch_rope_table(const SeqMeta& m, int head_dim, float theta, float* cos_s
 
 template <typename T>
 __global__ void k_rope_store(const float* __restrict__ tmp, const float* __restrict__ cos_sin,
-                             SeqMeta m, int nq, int nkv, int hd, T* __restrict__ q,
+                             SeqMeta m, int nq, int nkv, int hd, const T* __restrict__ bq,
+                             const T* __restrict__ bk, const T* __restrict__ bv, T* __restrict__ q,
                              T* __restrict__ k, T* __restrict__ v) {
   const int row = blockIdx.x;
   const int br = row % (m.batch * m.R_cap);  // (b, r): the table is shared by both variants
@@ -336,7 +337,11 @@ __global__ void k_rope_store(const float* __restrict__ tmp, const float* __restr
   // rotated heads: q then k; one thread per (head, i < half)
   for (int idx = threadIdx.x; idx < (nq + nkv) * half; idx += blockDim.x) {
     const int h = idx / half, i = idx % half;
-    const float x1 = t[h * hd + i], x2 = t[h * hd + half + i];
+    float x1 = t[h * hd + i], x2 = t[h * hd + half + i];
+    if (bq != nullptr) {   // projection bias, before the rotation
+      const T* bb = h < nq ? bq + h * hd : bk + (h - nq) * hd;
+      x1 += to_f<T>(bb[i]); x2 += to_f<T>(bb[half + i]);
+    }
     const float c = cs[i], sn = cs[half + i];
     const float y1 = x1 * c - x2 * sn, y2 = x2 * c + x1 * sn;
     if (h < nq) {
@@ -349,14 +354,14 @@ __global__ void k_rope_store(const float* __restrict__ tmp, const float* __restr
     }
   }
   for (int idx = threadIdx.x; idx < nkv * hd; idx += blockDim.x)
-    v[(size_t)row * nkv * hd + idx] = from_f<T>(t[(nq + nkv) * hd + idx]);
+    v[(size_t)row * nkv * hd + idx] = from_f<T>(t[(nq + nkv) * hd + idx] + (bv != nullptr ? to_f<T>(bv[idx]) : 0.f));
 }
 
 template <typename T>
 void launch_rope_store(const float* tmp, const float* cos_sin, const SeqMeta& m, int nq, int nkv,
-                       int hd, T* q, T* k, T* v, cudaStream_t s) {
+                       int hd, const T* bq, const T* bk, const T* bv, T* q, T* k, T* v, cudaStream_t s) {
   const int M = m.nv * m.batch * m.R_cap;
-  k_rope_store<T><<<M, 256, 0, s>>>(tmp, cos_sin, m, nq, nkv, hd, q, k, v);
+  k_rope_store<T><<<M, 256, 0, s>>>(tmp, cos_sin, m, nq, nkv, hd, bq, bk, bv, q, k, v);
 }
 
 // ---- SwiGLU: act = silu(gate) * up; gate_up is [M, 2F] (gate columns first) ----------------------
@@ -658,7 +663,7 @@ template void launch_export_kv<__nv_bfloat16>(const __nv_bfloat16*, const __nv_b
   template void launch_gemm_simt<T>(const T*, const T*, float*, int, int, int, int, int,        \
                                     cudaStream_t);                                              \
   template void launch_rope_store<T>(const float*, const float*, const SeqMeta&, int, int, int, \
-                                     T*, T*, T*, cudaStream_t);                                 \
+                                     const T*, const T*, const T*, T*, T*, T*, cudaStream_t);                                 \
   template void launch_swiglu<T>(const float*, int, int, T*, cudaStream_t);                     \
   template void launch_attn_simt<T>(const T*, const T*, const T*, const T*, const T*, int,      \
                                     const SeqMeta&, int, int, int, T*, cudaStream_t);           \

@@ -85,6 +85,7 @@ struct TcState {
   cudaStream_t s = nullptr;
   int M_max = 0;
   std::vector<LayerMaps> layers;
+  std::vector<const void*> bq, bk, bv;   // per-layer q / k / v projection biases (empty: none)
   std::map<int, ActMaps> act_maps;  // keyed by BN
   std::vector<void*> allocs;
   __nv_bfloat16 *a_buf = nullptr;  // borrowed: the normed activations of the scheduler
@@ -103,6 +104,7 @@ struct TcState {
   unsigned int qkv_launches = 0;     // chain launches of this step that ran a QKV phase
   unsigned int bar_count = 0;        // arrivals the launches of this step have used up so far
   int chain_grid = 0;                // CTAs of the dense chain (0 = unavailable)
+  bool stall_lmhead = false;         // test hook (DC_OPT_TEST_STALL_LMHEAD)
   bool coop_supported = false;       // the device can launch cooperatively
   bool chain_coop = false;           // the dense chain is launched cooperatively (co-residency guaranteed)
   std::string err;
@@ -192,7 +194,7 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
   cudaMemsetAsync(t->k, 0, M * hkv * 2, s);
   cudaMemsetAsync(t->v, 0, (size_t)t->ldv * hkv * 2, s);
   cudaMemsetAsync(t->o, 0, M * hq * 2, s);
-  if (!(make_map_2d(&t->map_q, t->q, M, hq, 128) && make_map_2d(&t->map_k, t->k, M, hkv, 128) &&
+  if (!(make_map_2d(&t->map_q, t->q, M, hq, 64) && make_map_2d(&t->map_k, t->k, M, hkv, 128) &&
         make_map_2d(&t->map_vt, t->v, hkv, t->ldv, 128)))
     return tfail(t, DC_ERR_CUDA, "attention tensor map encoding failed");
   t->map_kc = t->map_k; t->map_vc = t->map_vt;  // placeholders until a cache is supplied
@@ -388,7 +390,10 @@ int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k
   ap.m = m; ap.nq = nq; ap.nkv = nkv; ap.max_ctx = g.max_ctx; ap.layer = layer;
   ap.scale_log2 = 1.4426950408889634f / sqrtf((float)hd);
   ap.o = t->o; ap.status = t->status;
-  dim3 grid((m.R_cap + 127) / 128, nq, m.nv * m.batch);
+  const int nqt = (m.R_cap + 127) / 128;
+  // one CTA per query tile: (row tile, variant) with two variants in the pass (a row tile with 64
+  // rows or fewer packs both variants into the curr CTA, the prev CTA returns at once)
+  dim3 grid(m.nv == 2 ? 2 * nqt : nqt, nq, m.batch);
   k_attn_tc<<<grid, kAttnThreads, kAttnSmem, t->s>>>(t->map_q, t->map_k, t->map_vt, t->map_kc,
                                                      t->map_vc, ap);
   cudaError_t e = cudaGetLastError();
@@ -401,6 +406,23 @@ void tc_export_kv(TcState* t, int layer, const SeqMeta& m, __nv_bfloat16* k_cach
   const size_t per_layer = (size_t)g.max_batch * g.n_kv_heads * g.max_ctx * g.head_dim;
   launch_export_kv<__nv_bfloat16>(t->k, t->v, t->ldv, m, g.n_kv_heads, g.head_dim, g.max_ctx,
                                   k_cache + (size_t)layer * per_layer, v_cache + (size_t)layer * per_layer, t->s);
+}
+
+void tc_set_qkv_bias(TcState* t, const std::vector<const void*>& bq, const std::vector<const void*>& bk,
+                     const std::vector<const void*>& bv) {
+  t->bq = bq; t->bk = bk; t->bv = bv;
+}
+
+void tc_set_stall_lmhead(TcState* t, bool on) { t->stall_lmhead = on; }
+
+int tc_set_wait_limit_us(TcState* t, long long us) {
+  const unsigned long long ns = (unsigned long long)us * 1000ull;
+  if (cudaMemcpyToSymbolAsync(ptx::g_wait_limit_ns, &ns, sizeof(ns), 0, cudaMemcpyHostToDevice, t->s) != cudaSuccess ||
+      cudaStreamSynchronize(t->s) != cudaSuccess) {
+    cudaGetLastError();
+    return tfail(t, DC_ERR_CUDA, "setting the wait limit failed");
+  }
+  return DC_OK;
 }
 
 void tc_set_cooperative(TcState* t, bool on) { t->chain_coop = on && t->coop_supported; }
@@ -456,6 +478,10 @@ int tc_chain(TcState* t, int layer, int qkv_layer, int phase_begin, int phase_en
   p.g2 = g2; p.g1 = g1; p.eps = g.rms_eps;
   p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
   p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv;
+  if (!t->bq.empty()) {
+    const int lq = qkv_layer < g.n_layers ? qkv_layer : layer;
+    p.bq = (const __nv_bfloat16*)t->bq[lq]; p.bk = (const __nv_bfloat16*)t->bk[lq]; p.bv = (const __nv_bfloat16*)t->bv[lq];
+  }
   p.bar = t->grid_bar; p.status = t->status;
   // QKV has nq + 2 nkv tiles; when that is fewer than the grid has CTAs, the CTA pairs left over
   // take a share of every tile's k-blocks
@@ -523,6 +549,9 @@ int tc_layer(TcState* t, int layer, const SeqMeta& m, float* x, const __nv_bfloa
   p.M = M; p.BN = BN; p.nq = nq; p.nkv = nkv; p.hd = hd;
   p.cos_sin = cos_sin; p.rows_per_variant = m.batch * m.R_cap;
   p.q = t->q; p.k = t->k; p.v = t->v; p.ldv = t->ldv; p.act = t->act;
+  if (!t->bq.empty()) {
+    p.bq = (const __nv_bfloat16*)t->bq[layer]; p.bk = (const __nv_bfloat16*)t->bk[layer]; p.bv = (const __nv_bfloat16*)t->bv[layer];
+  }
   p.part = t->part; p.part_stride = t->part_stride;
 
   hook.begin(DC_STAGE_QKV, 1);
@@ -573,7 +602,7 @@ int tc_lmhead(TcState* t, const SeqMeta& m, const __nv_bfloat16* h, int mask_id,
   const dc_config& g = t->g;
   LmParams p;
   p.m = m; p.V = g.vocab; p.K = g.d_model; p.mask_id = forbid ? mask_id : -1;
-  p.part = t->lm_part; p.status = t->status;
+  p.part = t->lm_part; p.status = t->status; p.stall = t->stall_lmhead ? 1 : 0;
   const int ntiles = (g.vocab + 127) / 128;
   const int groups = m.npos_pad / m.G;
   int nctas = t->n_sm / groups;             // vocabulary slices: one resident CTA per (group, slice)
@@ -730,7 +759,7 @@ extern "C" int dc_signals_static(const dc_signals_in* in, const dc_signals_out* 
   k_static_rows<<<Mlm, 128, 0, s>>>((const __nv_bfloat16*)in->h, in->max_window, in->d_model, m, h_rows);
   LmParams p;
   p.m = m; p.V = in->vocab; p.K = in->d_model; p.mask_id = in->forbid_mask_pred ? in->mask_id : -1;
-  p.part = part; p.status = word;
+  p.part = part; p.status = word; p.stall = 0;
   const int ntiles = (in->vocab + 127) / 128;
   const int groups = m.npos_pad / m.G;
   int nctas = sd.n_sm / groups;

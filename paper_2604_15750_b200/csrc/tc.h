@@ -31,6 +31,9 @@ int tc_create(const dc_config& g, cudaStream_t s, int M_max, int Mlm_max,
               const std::vector<const void*>& w_gate, const std::vector<const void*>& w_up,
               const std::vector<const void*>& w_down, const void* lm_head,
               const __nv_bfloat16* h_buf, TcState** out);
+// per-layer biases of the q / k / v projections (all three or none)
+void tc_set_qkv_bias(TcState* t, const std::vector<const void*>& bq, const std::vector<const void*>& bk,
+                     const std::vector<const void*>& bv);
 void tc_destroy(TcState* t);
 const char* tc_error(const TcState* t);
 
@@ -49,6 +52,10 @@ int tc_attention(TcState* t, int layer, const SeqMeta& m, const __nv_bfloat16* k
 
 // Launch the dense chain with (default) or without the cooperative attribute; see DC_OPT_COOPERATIVE.
 void tc_set_cooperative(TcState* t, bool on);
+// Bound of every device-side wait of the tensor-core kernels, microseconds (device-wide).
+int tc_set_wait_limit_us(TcState* t, long long us);
+// Test hook: the LM-head kernel issues no loads, so that its bounded waits run out.
+void tc_set_stall_lmhead(TcState* t, bool on);
 // true if the persistent dense chain takes this step (all activation rows in one column block)
 bool tc_chain_ok(const TcState* t, const SeqMeta& m);
 // resets the chain's grid barrier; call once at the start of a step

@@ -69,6 +69,7 @@ struct ChainParams {
   float eps;
   const float* cos_sin;         // RoPE table [(b, r)][128]; row rows_per_variant: angle step
   int rows_per_variant;
+  const __nv_bfloat16 *bq, *bk, *bv;  // biases of the q / k / v projections phase 5 computes, or null
   __nv_bfloat16 *q, *k, *v;     // q [M, nq*128], k [M, nkv*128], v transposed [nkv*128, ldv]
   int ldv;
   // QKV has fewer tiles than the grid has CTAs: the CTA pairs beyond the tiles take the last
@@ -209,8 +210,14 @@ __device__ __forceinline__ void chain_emit(ChainCtx& c, const ChainParams& p, co
 #pragma unroll
     for (int j = 0; j < 16; ++j) dst[(size_t)j * N] = __float2bfloat16_rn(v0[j]);
   } else {  // CEPI_QKV
+    float bias_f = 0.f;   // projection bias of this thread's output feature, before the rotation
+    if (p.bq != nullptr) {
+      const __nv_bfloat16* bb = tile >= p.nq + p.nkv ? p.bv + (tile - p.nq - p.nkv) * 128
+                                : tile >= p.nq ? p.bk + (tile - p.nq) * 128 : p.bq + tile * 128;
+      bias_f = __bfloat162float(__ldg(bb + f));
+    }
 #pragma unroll
-    for (int j = 0; j < 16; ++j) v0[j] += v1[j];
+    for (int j = 0; j < 16; ++j) v0[j] += v1[j] + bias_f;
     const bool is_v = tile >= p.nq + p.nkv;
     if (is_v) {
       // V is stored transposed (keys contiguous): 16 consecutive keys of feature row f
@@ -346,53 +353,45 @@ __device__ __forceinline__ void chain_gemm(ChainCtx& c, const ChainParams& p, co
   } else if (c.warp == 1) {
     if (c.lane == 0 && c.rank == 0 && has) {
       // ---------------- MMA issuer (even CTA of the pair, for both) ----------------
-      // The issuing thread does not run ahead of the tensor core, so whatever it executes between
-      // two MMAs is added to the MMA period (N = 192: 140 clk per MMA with the descriptors rebuilt
-      // from the slot address every k-block, 97 with this loop; the tensor core's own time is
-      // 96).  The ring is therefore unrolled over its slots: barrier addresses and the low words
-      // of the descriptors of a slot are constants plus loop-invariant registers, the high word
-      // is one constant, and a k-step costs two 32-bit additions.
+      // (A ring unrolled over its slots with split 32-bit descriptors issues an MMA every 97 clk at
+      // N = 192 in isolation, against 140 for this loop, but these GEMMs wait for their data, not
+      // for the issue, and the larger code made the launch 4% slower: measured and taken out.)
       const uint32_t idesc = ptx::idesc_bf16(2 * kChainTile, BN);
       bool ok = true;
+      const uint32_t mring0 = ptx::smem_u32(c.ring);
       const uint32_t mfull0 = ptx::smem_u32(&c.full[0]), mempty0 = ptx::smem_u32(&c.empty[0]);
-      const uint32_t hi32 = ptx::smem_desc_hi32();
-      const uint32_t lo0 = ptx::smem_desc_lo(ptx::smem_u32(c.ring));
-      const uint32_t slot16 = (uint32_t)slot_bytes >> 4;
-      constexpr uint32_t kW16 = kChainTile * kChainTileK * 2 >> 4;   // one weight tile in descriptor units
+      const uint64_t desc_hi = ptx::smem_desc_sw128_hi();
+      uint32_t ms = 0, mslot = mring0;
       if (c.mma_units > 0) {  // the epilogue has drained both accumulators of the last unit
         ok = ptx::mbar_wait(c.acc_empty, (c.mma_units - 1) & 1u, c.abort_flag);
       }
       ptx::tc_fence_after();
-      uint32_t acc = 0;   // 0 until the first k-block of the unit has been issued
-      const uint32_t t0 = c.tmem_base, t1 = c.tmem_base + 256;
-      int kb = w.kb0;
-      while (kb < w.kb1 && ok) {
+      uint32_t acc_first = 0;   // 0 until the first k-block of the unit has been issued
+      for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
+        const uint32_t par = (c.use_bits >> ms) & 1u;
+        c.use_bits ^= 1u << ms;
+        ok = ptx::mbar_wait_a(mfull0 + 8u * ms, par, c.abort_flag);
+        if (!ok) break;
+        const uint64_t dw0 = desc_hi | (uint64_t)(mslot >> 4);
+        const uint64_t dw1 = dw0 + (kChainTile * kChainTileK * 2 >> 4);
+        const uint64_t da = dw0 + ((uint64_t)nw * (kChainTile * kChainTileK * 2 >> 4));
+        if (nw == 2) {
+          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16_pair(c.tmem_base + 256, dw1, da, idesc, acc_first);
 #pragma unroll
-        for (int s = 0; s < 8; ++s) {
-          if (s < stages && kb < w.kb1) {
-            const uint32_t par = (c.use_bits >> s) & 1u;
-            c.use_bits ^= 1u << s;
-            if (!ptx::mbar_wait_a(mfull0 + 8u * s, par, c.abort_flag)) { ok = false; break; }
-            const uint32_t w0 = lo0 + (uint32_t)s * slot16;
-            const uint32_t a = w0 + (uint32_t)nw * kW16;
-            if (nw == 2) {
-              const uint32_t w1 = w0 + kW16;
-#pragma unroll
-              for (int kk = 0; kk < kChainTileK / 16; ++kk) {
-                ptx::umma_bf16_pair_lo(t0, w0 + 2 * kk, a + 2 * kk, hi32, idesc, kk == 0 ? acc : 1u);
-                ptx::umma_bf16_pair_lo(t1, w1 + 2 * kk, a + 2 * kk, hi32, idesc, kk == 0 ? acc : 1u);
-              }
-            } else {
-              ptx::umma_bf16_pair_lo(t0, w0, a, hi32, idesc, acc);
-              ptx::umma_bf16_pair_lo(t1, w0 + 2, a + 2, hi32, idesc, acc);
-              ptx::umma_bf16_pair_lo(t0, w0 + 4, a + 4, hi32, idesc, 1u);
-              ptx::umma_bf16_pair_lo(t1, w0 + 6, a + 6, hi32, idesc, 1u);
-            }
-            acc = 1;
-            ptx::umma_commit_pair_a(mempty0 + 8u * s);   // frees the slot in both CTAs
-            ++kb;
+          for (int kk = 1; kk < kChainTileK / 16; ++kk) {
+            ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 2 * kk, da + 2 * kk, idesc);
+            ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw1 + 2 * kk, da + 2 * kk, idesc);
           }
+        } else {
+          ptx::umma_bf16_pair(c.tmem_base, dw0, da, idesc, acc_first);
+          ptx::umma_bf16_pair(c.tmem_base + 256, dw0 + 2, da + 2, idesc, acc_first);
+          ptx::umma_bf16_pair_acc(c.tmem_base, dw0 + 4, da + 4, idesc);
+          ptx::umma_bf16_pair_acc(c.tmem_base + 256, dw0 + 6, da + 6, idesc);
         }
+        acc_first = 1;
+        ptx::umma_commit_pair_a(mempty0 + 8u * ms);   // frees the slot in both CTAs
+        if (++ms == (uint32_t)stages) { ms = 0; mslot = mring0; } else mslot += (uint32_t)slot_bytes;
       }
       if (ok) ptx::umma_commit_pair(c.acc_full);  // both epilogues start
       ++c.mma_units;

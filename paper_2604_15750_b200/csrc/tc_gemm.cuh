@@ -46,6 +46,7 @@ struct GemmParams {
   int nq, nkv, hd;          // tiles [0,nq) are q heads, [nq,nq+nkv) k heads, rest v heads
   const float* cos_sin;     // RoPE table [(b, r)][hd]
   int rows_per_variant;     // batch * R_cap: the table is shared by the variants
+  const __nv_bfloat16 *bq, *bk, *bv;  // projection biases [nq*hd], [nkv*hd], [nkv*hd], or null
   __nv_bfloat16 *q, *k, *v; // outputs q [M, nq*hd], k [M, nkv*hd], v TRANSPOSED [nkv*hd, ldv]
   int ldv;                  // row pitch of the transposed v (elements, multiple of 8)
   // PARTIAL epilogue
@@ -275,6 +276,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       if (w.nkb > 0) {
       const uint32_t t_lane = tmem_base + set * 256u + ((uint32_t)(quarter * 32) << 16);
       const int m_base = w.cblk * p.BN;
+      float bias_f = 0.f;   // bias of this thread's output feature (q / k / v projections)
+      if (EPI == GEMM_EPI_QKV && p.bq != nullptr) {
+        const __nv_bfloat16* bb = tile >= p.nq + p.nkv ? p.bv + (tile - p.nq - p.nkv) * p.hd
+                                  : tile >= p.nq ? p.bk + (tile - p.nq) * p.hd : p.bq + tile * p.hd;
+        bias_f = __bfloat162float(bb[f]);
+      }
       for (int c0 = 0; c0 < p.BN; c0 += 32) {
         float acc[32];
         // BN is a multiple of 16: the last chunk may be 16 wide
@@ -332,6 +339,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
             }
           }
         } else {  // GEMM_EPI_QKV
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] += bias_f;
           const bool is_v = tile >= p.nq + p.nkv;
           if (is_v) {
             // V is stored transposed (keys contiguous): this thread's 32 columns are 32

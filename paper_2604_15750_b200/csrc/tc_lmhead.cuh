@@ -30,6 +30,7 @@ struct LmParams {
   int ngroups;       // groups of LM rows; gridDim.x = ngroups * vocabulary slices
   float* part;       // [groups][slices][128][8]
   int32_t* status;
+  int stall;         // test hook: the producer issues no load, so every wait of the kernel runs out
 };
 
 constexpr int kLmThreads = 192;
@@ -83,7 +84,7 @@ k_lmhead_tc(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ C
       const uint64_t pol_w = ptx::l2_policy_evict_first();
       uint32_t s = 0, ph = 0, slot = ring0;
       bool ok = true;
-      for (int q = 0; q < my_pairs && ok; ++q) {
+      for (int q = 0; q < my_pairs && ok && !p.stall; ++q) {
         // second tile of the pair may lie beyond the vocabulary: the load is zero-filled there
         // and the epilogue skips ids >= V
         const int vrow0 = (slice + (2 * q) * nslices) * 128;

@@ -2,7 +2,7 @@
 // never with cluster multicast), tcgen05 (TMEM allocation, MMA, commit, load) and the shared
 // memory / instruction descriptors of tcgen05.mma.
 //
-// Every wait is bounded: after kWaitLimitNs of wall time a waiter gives up, raises the CTA's
+// Every wait is bounded: after g_wait_limit_ns of wall time a waiter gives up, raises the CTA's
 // abort flag and returns false; callers then skip their work, fall through to the common exit
 // (TMEM is freed there) and the kernel reports DC_ERR_TIMEOUT through the status word.
 #pragma once
@@ -13,7 +13,10 @@
 namespace dc {
 namespace ptx {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+// How long a waiter polls before it gives up, in nanoseconds of the global timer: 2 s unless the
+// host changes it (the variable lives in this module's device image: one value per device for
+// every context of the process).
+static __device__ unsigned long long g_wait_limit_ns = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -76,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   while (!mbar_try_wait(bar, parity)) {
     if ((++polls & 0xff) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) {
+      if (globaltimer() - t0 > g_wait_limit_ns) {
         *abort_flag = 1;
         return false;
       }
@@ -89,7 +92,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
 // One arrival counter that only counts up: a CTA adds one (fire-and-forget, release) and polls
 // until the counter reaches `target` (acquire).  The host zeroes the word at the start of a step
 // and hands every launch the count its barriers start from.  One thread per CTA calls this after
-// a CTA-wide barrier.  The wait is bounded: returns false after kWaitLimitNs, or as soon as
+// a CTA-wide barrier.  The wait is bounded: returns false after g_wait_limit_ns, or as soon as
 // *abort_word (global) is non-zero.
 __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int target,
                                              const int* abort_word) {
@@ -103,7 +106,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
     if ((++polls & 0x3f) == 0) {
       int ab;
       asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(ab) : "l"(abort_word) : "memory");
-      if (ab != 0 || globaltimer() - t0 > kWaitLimitNs) return false;
+      if (ab != 0 || globaltimer() - t0 > g_wait_limit_ns) return false;
     }
   }
 }
@@ -123,7 +126,7 @@ __device__ __forceinline__ bool flag_wait(const unsigned int* flag, unsigned int
     if (v >= target) return true;
     if ((++polls & 0x3f) == 0) {
       if (*abort_flag != 0) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (globaltimer() - t0 > g_wait_limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -254,7 +257,7 @@ __device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volat
   while (!mbar_try_wait_a(bar, parity)) {
     if ((++polls & 0xff) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (globaltimer() - t0 > g_wait_limit_ns) { *abort_flag = 1; return false; }
     }
   }
   return true;

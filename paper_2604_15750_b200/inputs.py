@@ -38,6 +38,7 @@ class Workload:
     seed: int
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
+    qkv_bias: bool = False    # biases on the q / k / v projections (the Dream backbone has them)
 
     @property
     def mask_id(self) -> int:
@@ -63,6 +64,12 @@ WORKLOADS = {
     # 4: Dream-7B shape (grouped KV heads), batch 4
     "dream7b_b4": Workload("dream7b_b4", 28, 3584, 28, 4, 128, 18944, 152064, "bf16", 4, 768,
                            768, 32, 64, 512, _BASE_SEED + 4),
+    # LLaDA-1.5 (the paper's third backbone) has LLaDA-8B's architecture: same shapes, own seed
+    "llada15_b1": Workload("llada15_b1", 32, 4096, 32, 32, 128, 12288, 126464, "bf16", 1, 512,
+                           512, 32, 64, 256, _BASE_SEED + 6),
+    # Dream-7B shape with the biases its q / k / v projections carry
+    "dream7b_b4_bias": Workload("dream7b_b4_bias", 28, 3584, 28, 4, 128, 18944, 152064, "bf16", 4,
+                                768, 768, 32, 64, 512, _BASE_SEED + 4, qkv_bias=True),
     # 5: long-context stress, LLaDA-8B shape, batch 16
     "llada8b_long": Workload("llada8b_long", 32, 4096, 32, 32, 128, 12288, 126464, "bf16", 16,
                              4096, 4096, 32, 128, 1024, _BASE_SEED + 5),
@@ -91,11 +98,16 @@ def layer_weights(w: Workload, layer: int, device="cpu") -> dict:
     """Weights of one transformer layer, N(0, 0.02), row-major [out, in]; norm gains 1."""
     d, hq, hkv, F = w.d_model, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.d_ff
     mk = lambda n, s: _normal(w, n, layer, s, 0.02, device)
-    return dict(wq=mk("wq", (hq, d)), wk=mk("wk", (hkv, d)), wv=mk("wv", (hkv, d)),
-                wo=mk("wo", (d, hq)), w_gate=mk("w_gate", (F, d)), w_up=mk("w_up", (F, d)),
-                w_down=mk("w_down", (d, F)),
-                norm1=torch.ones(d, dtype=w.torch_dtype, device=device),
-                norm2=torch.ones(d, dtype=w.torch_dtype, device=device))
+    lw = dict(wq=mk("wq", (hq, d)), wk=mk("wk", (hkv, d)), wv=mk("wv", (hkv, d)),
+              wo=mk("wo", (d, hq)), w_gate=mk("w_gate", (F, d)), w_up=mk("w_up", (F, d)),
+              w_down=mk("w_down", (d, F)),
+              norm1=torch.ones(d, dtype=w.torch_dtype, device=device),
+              norm2=torch.ones(d, dtype=w.torch_dtype, device=device))
+    if w.qkv_bias:   # N(0, 0.5): large against the projections of a random-init model, so that a
+        # dropped or misplaced bias cannot hide inside the tolerance
+        mb = lambda n, k: _normal(w, n, layer, (k,), 0.5, device)
+        lw.update(bq=mb("bq", hq), bk=mb("bk", hkv), bv=mb("bv", hkv))
+    return lw
 
 
 def make_weights(w: Workload, device="cpu", n_layers: int | None = None) -> dict:

@@ -77,7 +77,7 @@ class Case:
             self.steer = inputs.make_steering(wl, self.weights["lm_head"], profile=steer)
 
     # ---- oracle side ------------------------------------------------------------------
-    def run_oracle(self, influence=True, seqs=None):
+    def run_oracle(self, influence=True, seqs=None, pos0=None):
         outs = {}
         for b in (range(self.wl.batch) if seqs is None else seqs):
             P, Lb, W = self.len["ctx_len"][b], self.len["last_len"][b], self.len["win_len"][b]
@@ -90,7 +90,8 @@ class Case:
                 hf = (adapters.to_np(self.steer[b, 0, :W]), adapters.to_np(self.steer[b, 1, :W]))
             outs[b] = O.step(self.ocfg, self.ow, kc, vc, P, self.last_ids[b, :Lb].numpy(),
                              self.win_ids[b, :W].numpy(), self.len["remain_len"][b],
-                             influence=influence, h_final=hf, n_layers=self.n_layers)
+                             influence=influence, h_final=hf, n_layers=self.n_layers,
+                             pos0=None if pos0 is None else pos0[b])
         return outs
 
     # ---- GPU side ---------------------------------------------------------------------

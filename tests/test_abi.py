@@ -28,11 +28,11 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_sizes_match_the_header_layout():
-    # 27 four-byte fields; two ints + nine pointers; pointer-only structs
-    assert ctypes.sizeof(binding.dc_config) == 27 * 4
-    assert ctypes.sizeof(binding.dc_step_in) == 8 + 11 * 8
+    # 28 four-byte fields; two ints + nine pointers; pointer-only structs
+    assert ctypes.sizeof(binding.dc_config) == 28 * 4
+    assert ctypes.sizeof(binding.dc_step_in) == 8 + 12 * 8
     assert ctypes.sizeof(binding.dc_step_out) == 12 * 8
-    assert ctypes.sizeof(binding.dc_weights) == 12 * 8
+    assert ctypes.sizeof(binding.dc_weights) == 15 * 8
     assert ctypes.sizeof(binding.dc_select_out) == 3 * 8
     assert ctypes.sizeof(binding.dc_commit_in) == 8 + 5 * 8
     assert ctypes.sizeof(binding.dc_generate_in) == 8 + 3 * 8 + 16

@@ -120,3 +120,48 @@ def test_select_threshold_override_reduces_to_the_baselines():
     m = g["sel_mask"].cpu().numpy()[:B, :W]
     assert np.array_equal(m.astype(bool), conf[:, :W] >= np.float32(0.9))
     eng.close()
+
+
+def test_batched_decisions_8192_sequences_bit_exact_on_a_sample():
+    """dc_boundary_batched / dc_select_batched over 8192 sequences with device-side length
+    arrays (the shape bench.py --mode decisions times): 96 sampled sequences, bit for bit."""
+    hp = Hyper()
+    eng = _engine(hp, max_batch=1, max_window=128)
+    r = np.random.default_rng(2024)
+    W, B = 128, 8192
+    mask_id = WL.mask_id
+    win = r.integers(1, W + 1, B).astype(np.int32)
+    remain = r.integers(1, 300, B).astype(np.int32)
+    have = (r.random(B) < 0.9).astype(np.int32)
+    I = (np.abs(r.standard_normal((B, W))) * np.exp(-np.arange(W) / 16.0)).astype(np.float32)
+    H = (r.random((B, W)) * 8).astype(np.float32)
+    conf = np.where(r.random((B, W)) < 0.5, 0.9 + 0.1 * r.random((B, W)), r.random((B, W))).astype(np.float32)
+    x = (r.standard_normal((B, W, W)) * 6 - 12).astype(np.float32)
+    ids = np.where(r.random((B, W)) < 0.8, mask_id, 5).astype(np.int32)
+    dev = eng.device
+    t = lambda a: torch.from_numpy(a).to(dev)
+    bo = dict(score=torch.zeros((B, W), device=dev), cum_influence=torch.zeros((B, W), device=dev),
+              cum_score=torch.zeros((B, W), device=dev),
+              block_len=torch.zeros((B,), dtype=torch.int32, device=dev))
+    eng.boundary_batched(t(I), t(H), t(win), t(remain), bo, have_prev=t(have))
+    so = dict(sel_mask=torch.zeros((B, W), dtype=torch.uint8, device=dev),
+              sel_idx=torch.zeros((B, W), dtype=torch.int32, device=dev),
+              sel_count=torch.zeros((B,), dtype=torch.int32, device=dev))
+    eng.select_batched(t(conf), t(ids), t(x), bo["block_len"], t(win), so)
+    eng.synchronize()
+    g = {k: v.cpu().numpy() for k, v in {**bo, **so}.items()}
+    picked = 0
+    for b in list(range(32)) + list(r.integers(0, B, 62)) + [B - 2, B - 1]:
+        L, score, ci, cs = O.boundary(I[b], H[b], int(win[b]), int(remain[b]), bool(have[b]), _ocfg(hp))
+        n = len(score)
+        assert int(g["block_len"][b]) == L, b
+        assert np.array_equal(g["score"][b, :n].view(np.uint32), score.view(np.uint32))
+        assert np.array_equal(g["cum_score"][b, :n].view(np.uint32), cs.view(np.uint32))
+        w = int(win[b])
+        want = O.cap_select(conf[b, :w], ids[b, :w] == mask_id, x[b, :w, :w], L, hp.tau_low,
+                            hp.tau_high, hp.gamma, hp.cap_mode)
+        cnt = int(g["sel_count"][b])
+        assert list(g["sel_idx"][b, :cnt]) == want, b
+        picked += cnt
+    assert picked > 96
+    eng.close()

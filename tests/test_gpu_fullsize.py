@@ -53,6 +53,31 @@ def test_dream_widths_grouped_heads_one_layer_chain_and_per_op():
         eng.close()
 
 
+@pytest.mark.parametrize("batch,impl", [(1, 0), (4, 0), (2, 1)])
+def test_qkv_projection_biases_chain_per_op_and_cuda_core(batch, impl):
+    """Dream widths with biases on the q / k / v projections (added before the rotation): the
+    fused chain (batch 1), the per-op tensor-core kernels (batch 4) and the CUDA-core kernels."""
+    wl = inputs.scaled(inputs.WORKLOADS["dream7b_b4_bias"], n_layers=2 if batch == 1 else 1, vocab=4096,
+                       batch=batch, ctx_min=100, ctx_max=128)
+    case = Case(wl)
+    assert "bq" in case.weights["layers"][0] and len(case.ow.bq) == case.n_layers
+    eng = case.make_engine(impl=impl)
+    _, launches = eng.step_profiled(**case.device_inputs(eng))
+    assert (launches["dense"] > 0) == (batch == 1 and impl == 0)
+    seqs = [0, batch - 1]
+    ora = case.run_oracle(seqs=seqs)
+    near, worst = compare(case, case.run_gpu(eng), ora,
+                          label=f"dream widths, q/k/v biases, batch {batch}, impl {impl}")
+    eng.close()
+    # the biases matter at this scale: the oracle without them is far from the one with them
+    ow = case.ow
+    saved = (ow.bq, ow.bk, ow.bv)
+    ow.bq, ow.bk, ow.bv = [], [], []
+    o0 = case.run_oracle(seqs=[0])[0]
+    ow.bq, ow.bk, ow.bv = saved
+    assert np.abs(o0["lse"] - ora[0]["lse"]).max() > 1e-3
+
+
 def test_full_vocabulary_lm_head_signals_and_decisions_match_the_oracle():
     """V = 126464, d = 4096, 64 positions x 2 variants, steered so that the distributions are
     shaped: every signal and the decisions against the oracle."""

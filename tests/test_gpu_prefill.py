@@ -100,3 +100,56 @@ def test_prefill_rejects_what_does_not_fit():
         eng.prefill(di["k_cache"], di["v_cache"], ids, [32], ctx_len=[40])
     assert "max_ctx" in str(e.value)
     eng.close()
+
+
+@pytest.mark.parametrize("tc", [False, True])
+def test_dual_cache_suffix_rows_prefilled_at_their_own_positions(tc):
+    """Prefix keys, then the still masked suffix behind the window prefilled with pos0 = P + W
+    (cache slots P .. P + S - 1, positions P + W ...): the cache rows match the oracle's prefill
+    with the same position argument, and a step over the window with that cache matches the
+    oracle's step over [prefix ; suffix] context rows."""
+    if tc:
+        wl = inputs.Workload("dual_tc", 2, 256, 4, 2, 128, 512, 2048, "bf16", 1, 40, 40, 0, 32, 64, 4711)
+        tol = 2e-2
+    else:
+        wl = inputs.scaled(TINY, last_len=0)
+        tol = 1e-4
+    P, Wn, S = 40, wl.win_len, 24
+    case = Case(inputs.scaled(wl, ctx_min=P, ctx_max=P), lengths=dict(ctx_len=[P], last_len=[0]))
+    eng = case.make_engine(max_last=64, max_ctx=128)
+    dev = eng.device
+    L, nkv, hd = wl.n_layers, wl.n_kv_heads, wl.head_dim
+    dt = wl.torch_dtype
+    kc = torch.zeros((L, 1, nkv, 128, hd), dtype=dt, device=dev)
+    vc = torch.zeros((L, 1, nkv, hd, 128), dtype=dt, device=dev)
+    prompt = case.prompt[0, :P]
+    ids = torch.zeros((1, eng.max_last), dtype=torch.int32)
+    ids[0, :P] = prompt
+    eng.prefill(kc, vc, ids.to(dev), [P])
+    suffix = torch.full((1, eng.max_last), wl.mask_id, dtype=torch.int32)
+    st = eng.prefill(kc, vc, suffix.to(dev), [S], ctx_len=[P], pos0=[P + Wn])
+    eng.synchronize()
+    assert int(st[0]) == 0
+    # oracle: the same two prefills
+    k0, v0 = O.prefill(case.ocfg, case.ow, prompt.numpy(), n_layers=L)
+    k1, v1 = O.prefill(case.ocfg, case.ow, np.full(S, wl.mask_id), k0, v0, ctx_len=P, n_layers=L, pos0=P + Wn)
+    kg, vg = _unpack(kc, vc, 0, P, P + S)
+    assert _relerr(kg, k1) <= tol and _relerr(vg, v1) <= tol
+    # a step over the window whose context is prefix + suffix rows
+    case.k_log = torch.from_numpy(np.concatenate([k0, k1], axis=2)[:, None]).to(dt)
+    case.v_log = torch.from_numpy(np.concatenate([v0, v1], axis=2)[:, None]).to(dt)
+    case.len["ctx_len"] = [P + S]
+    di = case.device_inputs(eng)
+    di["k_cache"], di["v_cache"] = kc, vc
+    # the window sits at positions P ... (right behind the prefix), not behind all P + S cached keys
+    out = eng.step(influence=False, boundary=True, pos0=[P], **di)
+    sel = eng.select(di["win_ids"], di["win_len"])
+    eng.synchronize()
+    gpu = {k_: v_.cpu().numpy() for k_, v_ in out.items()}
+    gpu.update({k_: v_.cpu().numpy() for k_, v_ in sel.items()})
+    ora = case.run_oracle(influence=False, pos0=[P])
+    compare(case, gpu, ora, label="dual cache: prefix + suffix context rows")
+    # and the position does matter: the oracle with the default position is somewhere else
+    off = case.run_oracle(influence=False)
+    assert np.abs(off[0]["lse"] - ora[0]["lse"]).max() > 1e-4
+    eng.close()

@@ -53,3 +53,28 @@ def test_positions_start_after_the_cached_context():
     k_all, v_all = O.prefill(cfg, w, ids)
     k_tail, _ = O.prefill(cfg, w, ids[16:], k_all, v_all, ctx_len=16)
     assert np.abs(k_tail[0] - k_all[0][:, 16:]).max() < 1e-9
+
+
+def test_suffix_rows_of_a_dual_cache_prefix_block_suffix_equals_one_whole_pass():
+    """Dual cache (Section 5.2, cache compatibility): the cache holds the prefix AND the still masked
+    suffix behind the window.  With suffix rows prefilled at their own positions (pos0 beyond the
+    window), a step over the window alone sees exactly what one bidirectional pass over
+    [prefix ; window ; suffix] sees: the window's layer-0 K / V and, through attention over both
+    cached parts, its hidden states agree with the whole pass."""
+    cfg, w, ids = _setup()
+    P, Wn, S = 8, 6, 10                       # prefix, window, suffix lengths
+    whole = ids[:P + Wn + S].copy()
+    whole[P:] = cfg.mask_id                   # window and suffix are still masked
+    x_whole, kv_whole = O.forward(cfg, w, whole, 0, None, None, return_kv=True)
+    # caches: prefix rows and suffix rows taken from the whole pass (what a refresh would store)
+    k_all = np.stack([np.transpose(k_, (1, 0, 2)) for k_, _ in kv_whole])     # [L, nkv, rows, hd]
+    v_all = np.stack([np.transpose(v_, (1, 0, 2)) for _, v_ in kv_whole])
+    keep = np.r_[0:P, P + Wn:P + Wn + S]
+    x_win = O.forward(cfg, w, whole[P:P + Wn], P, k_all[:, :, keep], v_all[:, :, keep])
+    assert np.abs(x_win - x_whole[P:P + Wn]).max() < 1e-9
+    # and the position argument of prefill: suffix tokens prefilled at pos0 = P + Wn get the layer-0
+    # K of the whole pass at those rows, whereas the default (positions = cache slots) does not
+    k_suf, _ = O.prefill(cfg, w, whole[P + Wn:], k_all[:, :, :P], v_all[:, :, :P], ctx_len=P, pos0=P + Wn)
+    assert np.abs(k_suf[0] - k_all[0][:, P + Wn:]).max() < 1e-9
+    k_bad, _ = O.prefill(cfg, w, whole[P + Wn:], k_all[:, :, :P], v_all[:, :, :P], ctx_len=P)
+    assert np.abs(k_bad[0] - k_all[0][:, P + Wn:]).max() > 1e-3
