@@ -386,6 +386,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b_b1", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="debug: run fewer layers (invalid as a result)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="debug: run fewer sequences of the workload (invalid as a result; for profiler captures)")
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-coop", action="store_true",
@@ -410,6 +412,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = inputs.WORKLOADS[args.workload]
+    if args.batch:
+        wl = inputs.scaled(wl, batch=args.batch)
     if args.impl == "reference":
         run_reference(args, wl, rank, world)
         return

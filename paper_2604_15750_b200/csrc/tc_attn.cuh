@@ -8,20 +8,22 @@
 // context tile between the variants and masks, per row, the active keys of the other variant.
 //
 // Per key tile:
-//   S = Q K^T        tcgen05.mma, fp32 in TMEM (two buffers of 128 columns)
+//   S = Q K^T        tcgen05.mma, fp32 in TMEM (three buffers of 128 columns)
 //   P = exp2(S - m)  softmax warps: thread <-> (row, quarter of the keys); the scores are read from
 //                    TMEM once, the probabilities go back into TMEM as packed bf16 over the
 //                    thread's own score columns
 //   O += P V         tcgen05.mma with the A operand in TMEM, accumulating over all tiles
-// S is double-buffered, so S of tile t+1 is computed while the softmax of tile t runs.  The
+// S has three buffers and runs two tiles ahead, so the softmax never waits for the scores: with
+// two buffers S of tile t + 2 could only start after P V of tile t, i.e. after the softmax of tile
+// t, and the period was half of (softmax + issue of both MMA groups) plus the load waits.  The
 // running maximum m only moves when a tile exceeds it by more than 2^8 (then the row's own
 // threads rescale O in TMEM).  Keys beyond the valid length are masked to -inf in S, and the V^T
 // columns of cached keys beyond ctx_len are zeroed in shared memory (the cache may hold anything
 // there).
 //
 // Warp roles (640 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + MMA issuer,
-// warp 2 = TMA producer for V^T, warp 3 = clears V^T columns beyond ctx_len and hands the slot to
-// the MMA issuer, warps 4..19 = softmax / output: four threads per row (TMEM lane quarter = warp
+// warp 2 = TMA producer for V^T, warp 3 = clears V^T columns beyond ctx_len, hands the slot to the
+// MMA issuer and, once P V has read it, back to the producer, warps 4..19 = softmax / output: four threads per row (TMEM lane quarter = warp
 // % 4), one for each quarter of a tile's keys and of O's columns.
 #pragma once
 #include "kernels.h"
@@ -117,10 +119,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const __grid_constant__ CUtensorMap map_vc, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, k_full[kAttnStagesK], k_empty[kAttnStagesK], v_loc[kAttnStagesV],
-      v_full[kAttnStagesV], v_empty[kAttnStagesV], s_full[2], p_full[2], pv_done[2], o_done;
+      v_full[kAttnStagesV], v_empty[kAttnStagesV], s_full[3], p_full[3], pv_done[3], o_done;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
-  __shared__ float xchg[4][128];   // [key quarter][row]: row maximum / row sum of each quarter
+  __shared__ float xchg[2][4][128];   // [tile parity][key quarter][row]: row maximum / row sum of each quarter
 
   const int b = blockIdx.z, h = blockIdx.y;
   AttnUnit un;
@@ -143,7 +145,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     for (int i = 0; i < kAttnStagesV; ++i) {
       ptx::mbar_init(&v_loc[i], 1); ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 3; ++i) {
       ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&p_full[i], 16); ptx::mbar_init(&pv_done[i], 1);
     }
     ptx::mbar_init(&o_done, 1);
@@ -157,7 +159,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  // TMEM columns: S / P of even tiles 0..127, of odd tiles 128..255, O 256..383
+  // TMEM columns: S / P of tile j in buffer j % 3 (columns 0..127, 128..255, 256..383), O 384..511
 
   if (warp == 0) {
     if (lane == 0) {
@@ -226,9 +228,16 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   } else if (warp == 3) {
     // ---------------- V^T slots: zero the columns of cached keys beyond ctx_len, then hand over ----
     bool ok = true;
+    static_assert(kAttnStagesV == 2, "the slot of tile j is the slot of tile j - 2");
     for (int j = 0; j < T && ok; ++j) {
       const int s = j % kAttnStagesV;
       const AttnTile t = attn_tile(un, j);
+      if (j >= kAttnStagesV) {
+        // P V of the tile that used this slot is complete: the producer may refill it
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done[(j - 2) % 3], ((uint32_t)(j - 2) / 3u) & 1u, &abort_flag));
+        if (!ok) break;
+        if (lane == 0) ptx::mbar_arrive(&v_empty[s]);
+      }
       ok = __all_sync(0xffffffffu, ptx::mbar_wait(&v_loc[s], ((uint32_t)(j / kAttnStagesV)) & 1u, &abort_flag));
       if (!ok) break;
       if (t.is_ctx && t.valid < kBK) {
@@ -255,15 +264,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(Ks));
       const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(Vs));
       constexpr uint32_t kSub16 = kSub >> 4;
-      const uint32_t b_k_full = ptx::smem_u32(&k_full[0]), b_k_empty = ptx::smem_u32(&k_empty[0]);
-      const uint32_t b_v_full = ptx::smem_u32(&v_full[0]), b_v_empty = ptx::smem_u32(&v_empty[0]);
+      const uint32_t b_k_full = ptx::smem_u32(&k_full[0]);
+      const uint32_t b_v_full = ptx::smem_u32(&v_full[0]);
       const uint32_t b_v_loc = ptx::smem_u32(&v_loc[0]);
       const uint32_t b_s_full = ptx::smem_u32(&s_full[0]), b_p_full = ptx::smem_u32(&p_full[0]);
       const uint32_t b_pv_done = ptx::smem_u32(&pv_done[0]);
-      // S(tile j) = Q K^T into score buffer j & 1.  The buffer last held P of tile j - 2, whose P V
+      // S(tile j) = Q K^T into score buffer j % 3.  The buffer last held P of tile j - 3, whose P V
       // was issued before this call: the tensor core runs its MMAs in issue order.
       auto issue_qk = [&](int j) {
-        const uint32_t s = (uint32_t)(j % kAttnStagesK), sb = (uint32_t)j & 1u;
+        const uint32_t s = (uint32_t)(j % kAttnStagesK), sb = (uint32_t)j % 3u;
         if (!ptx::mbar_wait_a(b_k_full + 8u * s, ((uint32_t)(j / kAttnStagesK)) & 1u, &abort_flag)) return false;
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + sb * 128u, bk = k_lo + s * (2 * kSub16);
@@ -272,20 +281,22 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const uint32_t off = (uint32_t)(kk >> 2) * kSub16 + (uint32_t)(kk & 3) * 2u;
           ptx::umma_bf16_lo(d, q_lo + off, bk + off, hi32, idesc, kk > 0 ? 1u : 0u);
         }
+        // (a commit costs the issuing thread about as much as three MMAs: the ring slots are handed
+        // back by other warps - K by a softmax thread that has seen S, V^T by the clearing warp
+        // that has seen P V complete)
         ptx::umma_commit_a(b_s_full + 8u * sb);
-        ptx::umma_commit_a(b_k_empty + 8u * s);   // the K slot is free once S is there
         return true;
       };
       // O (+)= P V; P sits in the score columns of its threads: keys 32 q + 2 c, + 1 in column 32 q + c
       auto issue_pv = [&](int j) {
         const uint32_t s = (uint32_t)(j % kAttnStagesV), ph = ((uint32_t)(j / kAttnStagesV)) & 1u;
-        const uint32_t sb = (uint32_t)j & 1u;
-        if (!ptx::mbar_wait_a(b_p_full + 8u * sb, ((uint32_t)j >> 1) & 1u, &abort_flag)) return false;
+        const uint32_t sb = (uint32_t)j % 3u;
+        if (!ptx::mbar_wait_a(b_p_full + 8u * sb, ((uint32_t)j / 3u) & 1u, &abort_flag)) return false;
         // the TMA's own barrier, then the hand-over of the clearing warp
         if (!ptx::mbar_wait_a(b_v_loc + 8u * s, ph, &abort_flag)) return false;
         if (!ptx::mbar_wait_a(b_v_full + 8u * s, ph, &abort_flag)) return false;
         ptx::tc_fence_after();
-        const uint32_t d = tmem_base + 256u, a = tmem_base + sb * 128u, bv = v_lo + s * (2 * kSub16);
+        const uint32_t d = tmem_base + 384u, a = tmem_base + sb * 128u, bv = v_lo + s * (2 * kSub16);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t off = (uint32_t)(kk >> 2) * kSub16 + (uint32_t)(kk & 3) * 2u;
@@ -293,13 +304,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
                                (kk > 0 || j > 0) ? 1u : 0u);
         }
         ptx::umma_commit_a(b_pv_done + 8u * sb);
-        ptx::umma_commit_a(b_v_empty + 8u * s);
         return true;
       };
       bool ok = ptx::mbar_wait(&q_full, 0, &abort_flag);
+      // the scores run two tiles ahead of the softmax: S of tile j + 2 is issued before P V of tile
+      // j waits for its probabilities
       if (ok) ok = issue_qk(0);
+      if (ok && T > 1) ok = issue_qk(1);
       for (int j = 0; j < T && ok; ++j) {
-        if (j + 1 < T) ok = issue_qk(j + 1);
+        if (j + 2 < T) ok = issue_qk(j + 2);
         if (ok) ok = issue_pv(j);
       }
       if (ok) ptx::umma_commit(&o_done);
@@ -311,7 +324,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     const int kq = gw >> 2;             // which 32 keys of a tile / which 32 columns of O
     const int r = quarter * 32 + lane;  // query row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t o_addr = t_lane + 256u + (uint32_t)kq * 32u;
+    const uint32_t o_addr = t_lane + 384u + (uint32_t)kq * 32u;
     const int kbase = kq * 32;
     const int my_variant = un.v[r >> 6];
     float m_run = -INFINITY, l_run = 0.f;   // l_run: this thread's keys only
@@ -323,12 +336,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     // partner warps waiting on a barrier.
     for (int j = 0; j < T; ++j) {
       const AttnTile t = attn_tile(un, j);
-      const uint32_t sb = (uint32_t)j & 1u;
+      const uint32_t sb = (uint32_t)j % 3u;
       const uint32_t s_addr = t_lane + sb * 128u + (uint32_t)kq * 32u;   // this thread's score columns
       // packed unit: an active key tile of the other variant contributes nothing to this warp's rows
       const bool other = un.packed && !t.is_ctx && t.kv != my_variant;
       const int nc = other ? 0 : max(0, min(32, t.valid - kbase));   // valid keys inside this thread's quarter
-      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], ((uint32_t)j >> 1) & 1u, &abort_flag));
+      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], ((uint32_t)j / 3u) & 1u, &abort_flag));
+      // S of this tile is complete, so its K slot has been read: hand it back to the producer
+      if (ok && gw == 0 && lane == 0) ptx::mbar_arrive(&k_empty[j % kAttnStagesK]);
       float sv[32];
       if (ok && nc > 0) {
         ptx::tc_fence_after();
@@ -349,10 +364,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         m2 = fmaxf(m2, sv[jj + 2]); m3 = fmaxf(m3, sv[jj + 3]);
       }
       float mx = ok ? fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) : -INFINITY;
-      xchg[kq][r] = mx;
+      // (two exchange buffers: the partners have passed the barrier of tile j + 1, hence read tile
+      // j's values, before anyone writes tile j + 2's)
+      float (*xc)[128] = xchg[j & 1];
+      xc[kq][r] = mx;
       row_sync();
-      mx = fmaxf(fmaxf(xchg[0][r], xchg[1][r]), fmaxf(xchg[2][r], xchg[3][r]));
-      row_sync();   // the partners have read before the next tile overwrites
+      mx = fmaxf(fmaxf(xc[0][r], xc[1][r]), fmaxf(xc[2][r], xc[3][r]));
       if (!ok) continue;
       const float m_tile = mx * p.scale_log2;
       // raise the running maximum only when the tile exceeds it by more than the gap
@@ -379,7 +396,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       m_run = m_new;
       if (j > 0 && __any_sync(0xffffffffu, raise)) {
         // O may be rescaled once P V of the tile before has completed
-        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done[sb ^ 1u], ((uint32_t)(j - 1) >> 1) & 1u, &abort_flag));
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done[(j - 1) % 3], ((uint32_t)(j - 1) / 3u) & 1u, &abort_flag));
         if (ok) {
           ptx::tc_fence_after();
           float ov[32];
@@ -397,9 +414,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     }
     if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_done, 0, &abort_flag));
     // row sum = the four quarters' sums
-    xchg[kq][r] = l_run;
+    float (*xl)[128] = xchg[T & 1];
+    xl[kq][r] = l_run;
     row_sync();
-    const float l_all = (xchg[0][r] + xchg[1][r]) + (xchg[2][r] + xchg[3][r]);
+    const float l_all = (xl[0][r] + xl[1][r]) + (xl[2][r] + xl[3][r]);
     const int hh = r >> 6, ri = r & 63;
     if (ok) {   // (the TMEM load is warp-wide: every lane takes part, valid row or not)
       ptx::tc_fence_after();
