@@ -326,6 +326,15 @@ __global__ void __launch_bounds__(kThreads) k_commit(int32_t* __restrict__ win_i
   }
 }
 
+__global__ void k_keep_block_len(int32_t* block_len, const PrevLen keep, int batch) {
+  const int b = threadIdx.x;
+  if (b < batch && keep.n[b] >= 0) block_len[b] = keep.n[b];
+}
+
+void launch_keep_block_len(int32_t* block_len, const PrevLen& keep, int batch, cudaStream_t s) {
+  k_keep_block_len<<<1, DC_MAX_BATCH, 0, s>>>(block_len, keep, batch);
+}
+
 void launch_commit(int32_t* win_ids, const int32_t* pred_id, const uint8_t* sel_mask,
                    const int32_t* block_len, const SeqMeta& m, int mask_id, int max_window,
                    int32_t* remaining, cudaStream_t s) {

@@ -92,6 +92,7 @@ struct dc_ctx {
   float *g_conf = nullptr, *g_xlogp = nullptr;
   char *g_hout = nullptr, *g_carry = nullptr;   // LM-head rows of a boundary step / kept for the next one
   uint8_t* g_mask = nullptr;
+  int32_t* g_host = nullptr;   // pinned: what a generation step reads back (block_len, remaining, status, window ids)
   SeqMeta last_meta{};
   bool have_logits = false;
   Profiler prof;
@@ -699,8 +700,17 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
   const size_t row_bytes = (size_t)g.d_model * (c->bf16 ? 2 : 4);
   std::vector<int32_t> h_prevlen(B);
   std::vector<Seq> sq(B);
-  std::vector<int32_t> h_ctx(B), h_lastlen(B), h_winlen(B), h_remain(B), h_blk(B), h_rem(B);
+  std::vector<int32_t> h_ctx(B), h_lastlen(B), h_winlen(B), h_remain(B);
   std::vector<int32_t> h_win((size_t)B * MW), h_last((size_t)B * (g.max_last > 0 ? g.max_last : 1));
+  if (!c->g_host && cudaMallocHost(reinterpret_cast<void**>(&c->g_host),
+                                   sizeof(int32_t) * (size_t)g.max_batch * (3 + MW)) != cudaSuccess) {
+    cudaGetLastError();
+    c->g_host = nullptr;
+    return fail(c, DC_ERR_NOMEM, "pinned staging buffer of dc_generate");
+  }
+  // one read-back per forward: [block_len | remaining | status | window ids], then one wait
+  int32_t *h_blk = c->g_host, *h_rem = h_blk + g.max_batch, *h_status = h_rem + g.max_batch,
+          *h_ids = h_status + g.max_batch;
   for (int b = 0; b < B; ++b) sq[b] = Seq{in->ctx_len[b], 0, 0, 0, 0, 0};
   if (out->block_lens) memset(out->block_lens, 0, sizeof(int32_t) * (size_t)B * N);
   cudaStream_t s = c->stream;
@@ -755,12 +765,16 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
     if (rc != DC_OK) return rc;
     ++nfe;
     // sequences inside a block keep their block length; the boundary rule wrote the others'
-    for (int b = 0; b < B; ++b)
-      if (!(sq[b].done < N && sq[b].blk == 0)) {
-        const int32_t keep = sq[b].done >= N ? 1 : sq[b].blk;
-        // pageable source: the call returns once the value has been staged
-        cudaMemcpyAsync(c->g_blk + b, &keep, sizeof(int32_t), cudaMemcpyHostToDevice, s);
+    {
+      PrevLen keep{};
+      bool any_keep = false;
+      for (int b = 0; b < B; ++b) {
+        const bool at_boundary = sq[b].done < N && sq[b].blk == 0;
+        keep.n[b] = at_boundary ? -1 : (sq[b].done >= N ? 1 : sq[b].blk);
+        any_keep |= !at_boundary;
       }
+      if (any_keep) launch_keep_block_len(c->g_blk, keep, B, s);
+    }
     dc_select_in se{};
     se.batch = B; se.conf = c->g_conf; se.win_ids = c->g_win; se.xlogp = c->g_xlogp;
     se.block_len = c->g_blk; se.win_len = h_winlen.data();
@@ -771,10 +785,10 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
     dc_commit_out co{c->g_rem};
     rc = dc_commit(c, &ci, &co);
     if (rc != DC_OK) return rc;
-    cudaMemcpyAsync(h_blk.data(), c->g_blk, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
-    cudaMemcpyAsync(h_rem.data(), c->g_rem, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
-    std::vector<int32_t> h_status(B);
-    cudaMemcpyAsync(h_status.data(), c->g_status, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(h_blk, c->g_blk, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(h_rem, c->g_rem, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(h_status, c->g_status, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(h_ids, c->g_win, sizeof(int32_t) * (size_t)B * MW, cudaMemcpyDeviceToHost, s);
     if (cudaStreamSynchronize(s) != cudaSuccess) return fail(c, DC_ERR_CUDA, "stream sync failed in dc_generate");
     for (int b = 0; b < B; ++b)
       if (h_status[b] != DC_OK) return fail(c, h_status[b], "device-side status %d in sequence %d", h_status[b], b);
@@ -796,12 +810,9 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
                             cudaMemcpyDeviceToDevice, s);
         }
       }
-      if (h_rem[b] == 0) {                     // block complete: read its ids back
-        if (cudaMemcpyAsync(out->tokens + (size_t)b * N + q.done, c->g_win + (size_t)b * MW,
-                            sizeof(int32_t) * q.blk, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess)
-          return fail(c, DC_ERR_CUDA, "reading a finished block back failed");
-        memcpy(h_last.data() + (size_t)b * g.max_last, out->tokens + (size_t)b * N + q.done, sizeof(int32_t) * q.blk);
+      if (h_rem[b] == 0) {                     // block complete: its ids came back with the counters
+        memcpy(out->tokens + (size_t)b * N + q.done, h_ids + (size_t)b * MW, sizeof(int32_t) * q.blk);
+        memcpy(h_last.data() + (size_t)b * g.max_last, h_ids + (size_t)b * MW, sizeof(int32_t) * q.blk);
         q.last_len = q.blk;
         q.done += q.blk;
         q.blk = 0;
@@ -854,6 +865,7 @@ int dc_destroy(dc_ctx* c) {
   if (!c) return DC_OK;
   if (c->tc) tc_destroy(c->tc);
   for (void* p : c->allocs) cudaFree(p);
+  if (c->g_host) cudaFreeHost(c->g_host);
   delete c;
   return DC_OK;
 }

@@ -149,4 +149,8 @@ void launch_commit(int32_t* win_ids, const int32_t* pred_id, const uint8_t* sel_
                    const int32_t* block_len, const SeqMeta& m, int mask_id, int max_window,
                    int32_t* remaining, cudaStream_t s);
 
+// block_len[b] = keep.n[b] for every sequence with keep.n[b] >= 0 (the others keep what the
+// boundary rule wrote)
+void launch_keep_block_len(int32_t* block_len, const PrevLen& keep, int batch, cudaStream_t s);
+
 }  // namespace dc

@@ -21,10 +21,13 @@
 // columns of cached keys beyond ctx_len are zeroed in shared memory (the cache may hold anything
 // there).
 //
-// Warp roles (640 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + MMA issuer,
-// warp 2 = TMA producer for V^T, warp 3 = clears V^T columns beyond ctx_len, hands the slot to the
-// MMA issuer and, once P V has read it, back to the producer, warps 4..19 = softmax / output: four threads per row (TMEM lane quarter = warp
-// % 4), one for each quarter of a tile's keys and of O's columns.
+// Warp roles (640 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the
+// score MMAs (Q K^T), warp 2 = TMA producer for V^T, warp 3 = issuer of the output MMAs (P V; all
+// its lanes first clear the V^T columns beyond ctx_len in the one tile that has any), warps 4..19 =
+// softmax / output: four threads per row (TMEM lane quarter = warp % 4), one for each quarter of a
+// tile's keys and of O's columns.  Two issuing threads because one was the bottleneck: with its
+// four barrier waits and two commits per tile it needed about 2270 clocks per tile for MMAs that
+// keep the tensor pipe busy for 1024.
 #pragma once
 #include "kernels.h"
 #include "tc_ptx.cuh"
@@ -47,7 +50,8 @@ constexpr int kBK = 128;                       // keys per tile
 constexpr int kSub = 128 * 128;                // bytes of one [128 rows x 64 bf16] sub-tile
 constexpr int kAttnStagesK = 3, kAttnStagesV = 2;   // ring slots of K and of V^T
 constexpr int kAttnSmem = 2 * kSub /*Q*/ + kAttnStagesK * 2 * kSub + kAttnStagesV * 2 * kSub + 1024;
-constexpr int kAttnPrefetch = 4;               // context tiles the L2 prefetch runs ahead of the ring
+constexpr int kAttnPrefetch = 0;               // context tiles the L2 prefetch runs ahead of the tile after the ring
+                                               // (measured: 0 -> 1.36 ms, 4 -> 1.41 ms, 8 -> 1.46 ms on 4 x 4096 keys x 8 layers)
 constexpr float kRescaleGap = 8.f;             // log2 units the tile maximum may exceed m before m moves
 
 __device__ __forceinline__ float attn_ex2(float x) {
@@ -119,7 +123,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const __grid_constant__ CUtensorMap map_vc, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, k_full[kAttnStagesK], k_empty[kAttnStagesK], v_loc[kAttnStagesV],
-      v_full[kAttnStagesV], v_empty[kAttnStagesV], s_full[3], p_full[3], pv_done[3], o_done;
+      s_full[3], p_full[3], pv_done[3], o_done;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float xchg[2][4][128];   // [tile parity][key quarter][row]: row maximum / row sum of each quarter
@@ -142,9 +146,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     abort_flag = 0;
     ptx::mbar_init(&q_full, 1);
     for (int i = 0; i < kAttnStagesK; ++i) { ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1); }
-    for (int i = 0; i < kAttnStagesV; ++i) {
-      ptx::mbar_init(&v_loc[i], 1); ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1);
-    }
+    for (int i = 0; i < kAttnStagesV; ++i) ptx::mbar_init(&v_loc[i], 1);
     for (int i = 0; i < 3; ++i) {
       ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&p_full[i], 16); ptx::mbar_init(&pv_done[i], 1);
     }
@@ -211,7 +213,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         const int s = j % kAttnStagesV;
         const AttnTile t = attn_tile(un, j);
         prefetch_v(j + kAttnStagesV + kAttnPrefetch);
-        if (!ptx::mbar_wait(&v_empty[s], (((uint32_t)(j / kAttnStagesV)) & 1u) ^ 1u, &abort_flag)) break;
+        // the slot held tile j - 2: free once its P V has completed
+        if (j >= kAttnStagesV &&
+            !ptx::mbar_wait(&pv_done[(j - 2) % 3], ((uint32_t)(j - 2) / 3u) & 1u, &abort_flag)) break;
         uint8_t* dst = Vs + (size_t)s * 2 * kSub;
         ptx::mbar_expect_tx(&v_loc[s], 2 * kSub);
         if (t.is_ctx) {
@@ -225,55 +229,24 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 3) {
-    // ---------------- V^T slots: zero the columns of cached keys beyond ctx_len, then hand over ----
-    bool ok = true;
-    static_assert(kAttnStagesV == 2, "the slot of tile j is the slot of tile j - 2");
-    for (int j = 0; j < T && ok; ++j) {
-      const int s = j % kAttnStagesV;
-      const AttnTile t = attn_tile(un, j);
-      if (j >= kAttnStagesV) {
-        // P V of the tile that used this slot is complete: the producer may refill it
-        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&pv_done[(j - 2) % 3], ((uint32_t)(j - 2) / 3u) & 1u, &abort_flag));
-        if (!ok) break;
-        if (lane == 0) ptx::mbar_arrive(&v_empty[s]);
-      }
-      ok = __all_sync(0xffffffffu, ptx::mbar_wait(&v_loc[s], ((uint32_t)(j / kAttnStagesV)) & 1u, &abort_flag));
-      if (!ok) break;
-      if (t.is_ctx && t.valid < kBK) {
-        // 0 * (whatever the cache holds there, NaN included) must not reach O
-        uint8_t* base = Vs + (size_t)s * 2 * kSub;
-        for (int rr = lane; rr < 128; rr += 32)
-          for (int cc = t.valid; cc < kBK; ++cc) {
-            const int c6 = cc & 63;
-            *reinterpret_cast<uint16_t*>(base + (cc >> 6) * kSub + rr * 128 + (((c6 >> 3) ^ (rr & 7)) << 4) + (c6 & 7) * 2) = 0;
-          }
-        ptx::fence_proxy_async_smem();
-      }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&v_full[s]);
-    }
   } else if (warp == 1) {
     if (lane == 0) {
-      // ---------------- MMA issuer ----------------
+      // ---------------- issuer of S = Q K^T ----------------
       // Lean issue path (the issuing thread does not run ahead of the tensor core): descriptor low
       // words are kept in registers and advanced by 32-bit additions of constants.
       const uint32_t idesc = ptx::idesc_bf16(128, 128);
       const uint32_t hi32 = ptx::smem_desc_hi32();
       const uint32_t q_lo = ptx::smem_desc_lo(ptx::smem_u32(Qs));
       const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(Ks));
-      const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(Vs));
       constexpr uint32_t kSub16 = kSub >> 4;
-      const uint32_t b_k_full = ptx::smem_u32(&k_full[0]);
-      const uint32_t b_v_full = ptx::smem_u32(&v_full[0]);
-      const uint32_t b_v_loc = ptx::smem_u32(&v_loc[0]);
-      const uint32_t b_s_full = ptx::smem_u32(&s_full[0]), b_p_full = ptx::smem_u32(&p_full[0]);
+      const uint32_t b_k_full = ptx::smem_u32(&k_full[0]), b_s_full = ptx::smem_u32(&s_full[0]);
       const uint32_t b_pv_done = ptx::smem_u32(&pv_done[0]);
-      // S(tile j) = Q K^T into score buffer j % 3.  The buffer last held P of tile j - 3, whose P V
-      // was issued before this call: the tensor core runs its MMAs in issue order.
-      auto issue_qk = [&](int j) {
+      bool ok = ptx::mbar_wait(&q_full, 0, &abort_flag);
+      for (int j = 0; j < T && ok; ++j) {
         const uint32_t s = (uint32_t)(j % kAttnStagesK), sb = (uint32_t)j % 3u;
-        if (!ptx::mbar_wait_a(b_k_full + 8u * s, ((uint32_t)(j / kAttnStagesK)) & 1u, &abort_flag)) return false;
+        // score buffer j % 3 last held P of tile j - 3: its P V (issued by another thread) must be done
+        if (j >= 3 && !ptx::mbar_wait_a(b_pv_done + 8u * sb, ((uint32_t)(j - 3) / 3u) & 1u, &abort_flag)) break;
+        if (!ptx::mbar_wait_a(b_k_full + 8u * s, ((uint32_t)(j / kAttnStagesK)) & 1u, &abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + sb * 128u, bk = k_lo + s * (2 * kSub16);
 #pragma unroll
@@ -281,42 +254,60 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const uint32_t off = (uint32_t)(kk >> 2) * kSub16 + (uint32_t)(kk & 3) * 2u;
           ptx::umma_bf16_lo(d, q_lo + off, bk + off, hi32, idesc, kk > 0 ? 1u : 0u);
         }
-        // (a commit costs the issuing thread about as much as three MMAs: the ring slots are handed
-        // back by other warps - K by a softmax thread that has seen S, V^T by the clearing warp
-        // that has seen P V complete)
+        // (the K slot is handed back by a softmax thread that has seen S)
         ptx::umma_commit_a(b_s_full + 8u * sb);
-        return true;
-      };
-      // O (+)= P V; P sits in the score columns of its threads: keys 32 q + 2 c, + 1 in column 32 q + c
-      auto issue_pv = [&](int j) {
-        const uint32_t s = (uint32_t)(j % kAttnStagesV), ph = ((uint32_t)(j / kAttnStagesV)) & 1u;
-        const uint32_t sb = (uint32_t)j % 3u;
-        if (!ptx::mbar_wait_a(b_p_full + 8u * sb, ((uint32_t)j / 3u) & 1u, &abort_flag)) return false;
-        // the TMA's own barrier, then the hand-over of the clearing warp
-        if (!ptx::mbar_wait_a(b_v_loc + 8u * s, ph, &abort_flag)) return false;
-        if (!ptx::mbar_wait_a(b_v_full + 8u * s, ph, &abort_flag)) return false;
-        ptx::tc_fence_after();
-        const uint32_t d = tmem_base + 384u, a = tmem_base + sb * 128u, bv = v_lo + s * (2 * kSub16);
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (uint32_t)(kk >> 2) * kSub16 + (uint32_t)(kk & 3) * 2u;
-          ptx::umma_bf16_ts_lo(d, a + (uint32_t)(kk >> 1) * 32u + (uint32_t)(kk & 1) * 8u, bv + off, hi32, idesc,
-                               (kk > 0 || j > 0) ? 1u : 0u);
-        }
-        ptx::umma_commit_a(b_pv_done + 8u * sb);
-        return true;
-      };
-      bool ok = ptx::mbar_wait(&q_full, 0, &abort_flag);
-      // the scores run two tiles ahead of the softmax: S of tile j + 2 is issued before P V of tile
-      // j waits for its probabilities
-      if (ok) ok = issue_qk(0);
-      if (ok && T > 1) ok = issue_qk(1);
-      for (int j = 0; j < T && ok; ++j) {
-        if (j + 2 < T) ok = issue_qk(j + 2);
-        if (ok) ok = issue_pv(j);
       }
-      if (ok) ptx::umma_commit(&o_done);
     }
+  } else if (warp == 3) {
+    // ---------------- issuer of O (+)= P V ----------------
+    // P sits in the score columns of its threads: keys 32 q + 2 c, + 1 in column 32 q + c.
+    static_assert(kAttnStagesV == 2, "the slot of tile j is the slot of tile j - 2");
+    const uint32_t idesc = ptx::idesc_bf16(128, 128);
+    const uint32_t hi32 = ptx::smem_desc_hi32();
+    const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(Vs));
+    constexpr uint32_t kSub16 = kSub >> 4;
+    const uint32_t b_v_loc = ptx::smem_u32(&v_loc[0]), b_p_full = ptx::smem_u32(&p_full[0]);
+    const uint32_t b_pv_done = ptx::smem_u32(&pv_done[0]);
+    bool ok = true;
+    for (int j = 0; j < T && ok; ++j) {
+      const uint32_t s = (uint32_t)(j % kAttnStagesV), ph = ((uint32_t)(j / kAttnStagesV)) & 1u;
+      const uint32_t sb = (uint32_t)j % 3u;
+      const AttnTile t = attn_tile(un, j);
+      if (t.is_ctx && t.valid < kBK) {
+        // The one context tile with cached keys beyond ctx_len: all lanes zero those V^T columns
+        // (0 * whatever the cache holds there, NaN included, must not reach O).
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait_a(b_v_loc + 8u * s, ph, &abort_flag));
+        if (!ok) break;
+        uint8_t* base = Vs + (size_t)s * 2 * kSub;
+        for (int rr = lane; rr < 128; rr += 32)
+          for (int cc = t.valid; cc < kBK; ++cc) {
+            const int c6 = cc & 63;
+            *reinterpret_cast<uint16_t*>(base + (cc >> 6) * kSub + rr * 128 + (((c6 >> 3) ^ (rr & 7)) << 4) + (c6 & 7) * 2) = 0;
+          }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+      }
+      if (lane == 0) {
+        ok = ptx::mbar_wait_a(b_p_full + 8u * sb, ((uint32_t)j / 3u) & 1u, &abort_flag) &&
+             ptx::mbar_wait_a(b_v_loc + 8u * s, ph, &abort_flag);
+        if (ok) {
+          ptx::tc_fence_after();
+          const uint32_t d = tmem_base + 384u, a = tmem_base + sb * 128u, bv = v_lo + s * (2 * kSub16);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * kSub16 + (uint32_t)(kk & 3) * 2u;
+            ptx::umma_bf16_ts_lo(d, a + (uint32_t)(kk >> 1) * 32u + (uint32_t)(kk & 1) * 8u, bv + off, hi32, idesc,
+                                 (kk > 0 || j > 0) ? 1u : 0u);
+          }
+          // also tells the V^T producer that the slot is free, the score issuer that the buffer
+          // is, and the softmax warps that O may be rescaled
+          ptx::umma_commit_a(b_pv_done + 8u * sb);
+        }
+      }
+      // the other lanes wait here (not spinning) while lane 0 issues
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    }
+    if (ok && lane == 0) ptx::umma_commit(&o_done);
   } else {
     // ---------------- softmax / output warps ----------------
     const int gw = warp - 4;
