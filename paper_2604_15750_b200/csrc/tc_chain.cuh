@@ -20,10 +20,11 @@
 //
 // GEMM orientation (as in tc_gemm.cuh): a CTA owns 128 weight rows (MMA M, one TMEM lane per
 // output feature) and all activation rows (MMA N <= 256, one TMEM column per row).  Every unit
-// keeps TWO accumulators in flight, because a chain of tcgen05.mma into one accumulator issues
-// at 151 clk per MMA while two alternating accumulators reach max(86, N/2 + 21) clk: gate / up
-// use one accumulator each, the other GEMMs send even k-steps to the first and odd k-steps to the
-// second and add them in the epilogue.
+// keeps two accumulators: gate / up use one each, the other GEMMs send even k-steps to the first
+// and odd k-steps to the second and add them in the epilogue.  (The split is not what sets the
+// issue rate: a lean issue loop reaches the tensor core's own N / 2 clocks per pair MMA with one
+// accumulator chain as with two; what costs is every instruction the issuing thread executes
+// between two MMAs.  These GEMMs wait for their weights, not for the issue.)
 //
 // CTA pairs: the launch uses clusters of two CTAs and every MMA is a pair MMA (cta_group::2,
 // M = 256): each CTA streams its own 128 weight rows but only HALF of the activation rows, the

@@ -12,9 +12,10 @@
 // TMEM columns are 128 vocabulary entries, so each thread scans its own row serially; the only
 // exchange is z' from the prev row's thread to the curr row's thread, through shared memory.
 // CTAs are persistent over vocabulary tiles (tile = blockIdx.x, += gridDim.x), two tiles at a
-// time: the MMAs of a pair alternate between two TMEM accumulators (a chain of MMAs into one
-// accumulator issues at 151 clk per MMA, two alternating ones at 86 clk for N = 128, and both
-// MMAs of a k-step share the h operand), and two such pairs of accumulators exist, so that the
+// time: the MMAs of a pair alternate between two TMEM accumulators (both MMAs of a k-step share
+// the h operand; the issue rate is set by the instructions between two MMAs of the issuing
+// thread, not by the accumulator dependence: a lean loop reaches the tensor core's own 64 clk per
+// 128 x 128 x 16 MMA with one accumulator as with two), and two such pairs of accumulators exist, so that the
 // statistics of one pair overlap the MMAs of the next.  Each CTA writes one partial record per
 // row; k_lm_combine merges the records of all CTAs.
 #pragma once
