@@ -402,7 +402,8 @@ DC_API int dc_step_profiled(dc_ctx* ctx, const dc_step_in* in, const dc_step_out
  * DC_STATIC_MAX_POS positions, vocab >= 2.
  *
  * The first call on a device looks up the device address of the array and opts the kernel in to
- * its shared memory; make that first call before any stream capture.  All calls on a device
+ * its shared memory; make that first call before any stream capture, and from one host thread
+ * (the per-device address table is filled without a lock; later calls only read it).  All calls on a device
  * share the one array, which keeps the previous call's contents: the call itself clears what
  * must start at zero, but two calls whose kernels overlap on the GPU (different streams, no
  * dependency) race on it - order them.  The caller passes inputs and outputs as usual; outputs
