@@ -267,6 +267,7 @@ def run_generate(args, wl, dev):
     nb = [len(b) for b in blocks]
     print(json.dumps(dict(metric="generated_tokens_per_s", value=wl.batch * N / dt, unit="tokens/s",
                           n_gpus=1, mode="generate", ms=dt * 1e3, nfe=nfe,
+                          device_ms=eng.last_generate_device_ms, host_gap_ms=dt * 1e3 - eng.last_generate_device_ms,
                           tokens_per_forward=wl.batch * N / nfe, ms_per_forward=dt * 1e3 / nfe,
                           blocks_per_sequence=nb, mean_block_len=float(N * wl.batch / max(sum(nb), 1)),
                           dtype="bf16" if wl.dtype == "bf16" else "f32", data="synthetic",

@@ -335,6 +335,9 @@ typedef struct dc_generate_out {
   int32_t* tokens;           /* HOST [batch][gen_len]                                         */
   int32_t* block_lens;       /* HOST [batch][gen_len]: lengths of the blocks in order, then 0 */
   int32_t* nfe;              /* HOST [1]: dc_step calls made (model forward evaluations)      */
+  float* device_ms;          /* HOST [1] or null: summed device time of all forwards (CUDA events
+                                around each forward's launches); wall clock minus this is what the
+                                host loop and its read-backs cost                              */
 } dc_generate_out;
 DC_API int dc_generate(dc_ctx* ctx, const dc_generate_in* in, const dc_generate_out* out);
 

@@ -116,7 +116,7 @@ class dc_generate_in(C.Structure):
 
 
 class dc_generate_out(C.Structure):
-    _fields_ = [("tokens", _I32P), ("block_lens", _I32P), ("nfe", _I32P)]
+    _fields_ = [("tokens", _I32P), ("block_lens", _I32P), ("nfe", _I32P), ("device_ms", C.POINTER(C.c_float))]
 
 
 class dc_signals_in(C.Structure):
@@ -465,9 +465,11 @@ class DepCap:
         gi = dc_generate_in(batch=B, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
                             ctx_len=C.cast(cl_, _I32P), gen_len=gen_len, max_steps=max_steps,
                             carried_prev=int(carried_prev))
+        dev_ms = (C.c_float * 1)()
         go = dc_generate_out(tokens=C.cast(tokens, _I32P), block_lens=C.cast(blocks, _I32P),
-                             nfe=C.cast(nfe, _I32P))
+                             nfe=C.cast(nfe, _I32P), device_ms=C.cast(dev_ms, C.POINTER(C.c_float)))
         self._check(self._lib.dc_generate(self._ctx, C.byref(gi), C.byref(go)))
+        self.last_generate_device_ms = float(dev_ms[0])
         tok = np.ctypeslib.as_array(tokens).reshape(B, gen_len).copy()
         bl = np.ctypeslib.as_array(blocks).reshape(B, gen_len).copy()
         return tok, [[int(x) for x in row if x > 0] for row in bl], int(nfe[0])

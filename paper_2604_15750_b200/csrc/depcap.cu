@@ -715,6 +715,14 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
   if (out->block_lens) memset(out->block_lens, 0, sizeof(int32_t) * (size_t)B * N);
   cudaStream_t s = c->stream;
   int nfe = 0;
+  // device time of the forwards (optional): one pair of events, read after each forward's wait
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  double dev_ms = 0.0;
+  if (out->device_ms && (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess)) {
+    if (ev0) cudaEventDestroy(ev0);
+    return fail(c, DC_ERR_CUDA, "event creation failed in dc_generate");
+  }
+  struct EvGuard { cudaEvent_t &a, &b; ~EvGuard() { if (a) cudaEventDestroy(a); if (b) cudaEventDestroy(b); } } ev_guard{ev0, ev1};
   while (true) {
     bool any_open = false, any_boundary = false;
     for (int b = 0; b < B; ++b) {
@@ -723,6 +731,7 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
     }
     if (!any_open) break;
     if (nfe >= max_steps) { *out->nfe = nfe; return fail(c, DC_ERR_TIMEOUT, "max_steps=%d reached", max_steps); }
+    if (ev0) cudaEventRecord(ev0, s);
     // ---- inputs of this step
     for (int b = 0; b < B; ++b) {
       Seq& q = sq[b];
@@ -789,7 +798,12 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
     cudaMemcpyAsync(h_rem, c->g_rem, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
     cudaMemcpyAsync(h_status, c->g_status, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s);
     cudaMemcpyAsync(h_ids, c->g_win, sizeof(int32_t) * (size_t)B * MW, cudaMemcpyDeviceToHost, s);
+    if (ev1) cudaEventRecord(ev1, s);
     if (cudaStreamSynchronize(s) != cudaSuccess) return fail(c, DC_ERR_CUDA, "stream sync failed in dc_generate");
+    if (ev1) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ev0, ev1) == cudaSuccess) dev_ms += ms;
+    }
     for (int b = 0; b < B; ++b)
       if (h_status[b] != DC_OK) return fail(c, h_status[b], "device-side status %d in sequence %d", h_status[b], b);
     // ---- state update
@@ -820,6 +834,7 @@ int dc_generate(dc_ctx* c, const dc_generate_in* in, const dc_generate_out* out)
     }
   }
   *out->nfe = nfe;
+  if (out->device_ms) *out->device_ms = (float)dev_ms;
   return DC_OK;
 }
 

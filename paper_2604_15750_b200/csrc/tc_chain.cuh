@@ -93,17 +93,9 @@ constexpr int kChainXch = kChainParts * 128 * kXchRow * 4;  // RoPE exchange buf
 constexpr int kChainSmem = kChainRing + kChainXch + 1024;
 constexpr int kChainTile = 128;                 // weight rows per unit
 constexpr int kChainTileK = 64;
-// k-blocks of its next unit that a CTA prefetches into L2 when its own loads are issued
-#ifndef DC_PF_GU
-#define DC_PF_GU 4
-#endif
-#ifndef DC_PF_DN
-#define DC_PF_DN 4
-#endif
-#ifndef DC_PF_QKV
-#define DC_PF_QKV 4
-#endif
-constexpr int kPfGateUp = DC_PF_GU, kPfDown = DC_PF_DN, kPfQkv = DC_PF_QKV;
+// k-blocks of its next unit that a CTA prefetches into L2 when its own loads are issued (measured:
+// 8 / 12 / 24 k-blocks cost +0.03 / +0.04 / +0.25 ms per step against 4)
+constexpr int kPfGateUp = 4, kPfDown = 4, kPfQkv = 4;
 
 struct ChainCtx {
   uint8_t* ring;

@@ -36,7 +36,7 @@ def test_struct_sizes_match_the_header_layout():
     assert ctypes.sizeof(binding.dc_select_out) == 3 * 8
     assert ctypes.sizeof(binding.dc_commit_in) == 8 + 5 * 8
     assert ctypes.sizeof(binding.dc_generate_in) == 8 + 3 * 8 + 16
-    assert ctypes.sizeof(binding.dc_generate_out) == 3 * 8
+    assert ctypes.sizeof(binding.dc_generate_out) == 4 * 8
 
 
 def test_last_error_without_context_is_a_string():
