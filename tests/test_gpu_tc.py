@@ -78,6 +78,33 @@ def test_tc_more_than_128_active_rows_and_long_context():
     eng.close()
 
 
+def test_tc_attention_scores_far_above_those_of_the_first_key_tile():
+    """The attention kernel fixes a row's reference point from its first key tile and runs a second
+    pass when a later score lies more than 2^100 above it.  Three cached keys behind the first tile
+    are scaled by 2000: for the rows whose query points their way they dominate by hundreds of log2
+    units (one of them takes all the weight), for the others they vanish; with R = 160 active rows
+    both the one-variant tiles and the packed tile of both variants go through it."""
+    wl = _wl(2, ctx=(300, 300), last=32, win=128)
+    case = Case(wl)
+    for pos in (150, 210, 290):
+        case.k_log[:, :, :, pos, :] *= 2000.0
+    eng = case.make_engine()
+    gpu, ora = case.run_gpu(eng), case.run_oracle()
+    eng.close()
+    # Scores of several hundred log2 units turn a last-place difference in a rotated query into a
+    # visible shift of weight between two keys, so the difference of the two variants (I_k) is
+    # compared at 2e-2 absolute here instead of the 1e-3 of the well-conditioned cases; the
+    # per-variant quantities keep their usual tolerance.
+    for b in range(2):
+        W = case.len["win_len"][b]
+        for name in ("conf", "entropy", "lse"):
+            ref = ora[b][name]
+            err = np.abs(gpu[name][b, :W] - ref) / np.maximum(np.abs(ref), 1.0)
+            assert np.isfinite(gpu[name][b, :W]).all() and err.max() <= 2e-2, (name, b, err.max())
+        assert np.abs(gpu["influence"][b, :W] - ora[b]["influence"]).max() <= 2e-2
+        assert (gpu["pred_id"][b, :W] == ora[b]["pred"]).mean() >= 0.95
+
+
 def test_fused_dense_chain_is_the_path_taken_when_the_rows_fit_one_block():
     """M = 2 * 2 * 48 = 192 activation rows: the persistent dense chain must run (one launch that
     starts the step plus one per layer), not the per-op kernels; with 3 * 48 * 2 = 288 rows the
