@@ -14,7 +14,7 @@
 //   O += P V          tcgen05.mma with the A operand in TMEM, accumulating over all tiles
 //
 // The reference point m0 of a row is fixed for the whole pass: the row's maximum over the first
-// key tile (0 if that tile has no valid key for the row).  Floating point does not care how far
+// 32 keys of the first tile (0 if none of them is valid for the row).  Floating point does not care how far
 // the later scores lie from it as long as 2^(s - m0) stays in range; a pass in which some row's
 // running maximum ends more than 2^100 above its m0 is run again with m0 = that maximum (a CTA-wide
 // decision at the end of the pass; at most once).  With m0 fixed the tiles of a row are
@@ -355,20 +355,16 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         const int nvalid = (other || !sm_ok) ? 0 : t.valid;   // warp-uniform
         if (sm_ok) ptx::tc_fence_after();
         float sv[2][32];
+        if (nvalid > 0) ptx::tmem_ld_32x32(s_addr, sv[0]);   // the first 32 keys of the tile
         if (!have_m0) {
           if (J == 0) {
-            // this warp owns the first tile: its rows' maxima there are the rows' reference points
+            // this warp owns the first tile: the rows' maxima over its first 32 keys are the rows'
+            // reference points (any score of the row would do)
+            ptx::tmem_ld_wait();
+            const int nc = max(0, min(32, nvalid));
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const int nc = max(0, min(32, nvalid - 32 * c));
-              if (nc > 0) {
-                ptx::tmem_ld_32x32(s_addr + 32u * c, sv[0]);
-                ptx::tmem_ld_wait();
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) mx = fmaxf(mx, jj < nc ? sv[0][jj] : -INFINITY);
-              }
-            }
+            for (int jj = 0; jj < 32; ++jj) mx = fmaxf(mx, jj < nc ? sv[0][jj] : -INFINITY);
             m0 = mx == -INFINITY ? 0.f : mx * scale;
             m_row[r] = m0;
             __syncwarp();
@@ -383,7 +379,6 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         const ptx::f32x2 scale2 = ptx::f2_pack(scale, scale), negm2 = ptx::f2_pack(-m0, -m0);
         ptx::f32x2 la = ptx::f2_pack(0.f, 0.f), lb = la;
         float x0 = run_max, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
-        if (nvalid > 0) ptx::tmem_ld_32x32(s_addr, sv[0]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           float (&v)[32] = sv[c & 1];
