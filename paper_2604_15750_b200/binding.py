@@ -290,6 +290,12 @@ class DepCap:
                                      C.byref(self._ctx))
         if rc != DC_OK:
             raise DepCapError(rc, self._lib.dc_last_error(None).decode())
+        if "NV_COMPUTE_PROFILER_PERFWORKS_DIR" in os.environ:
+            # Running under Nsight Compute, which cannot replay a cooperative cluster launch (it ends
+            # the process with "LaunchFailed"): launch the dense chain without the attribute.  Same
+            # grid, same kernel; under the profiler nothing else runs on the GPU, so all CTAs are
+            # resident, and every wait in the kernel is bounded anyway.
+            self._lib.dc_set_option(self._ctx, DC_OPT_COOPERATIVE, 0)
         B, W = max_batch, max_window
         dev = self.device
         f = lambda *s: torch.zeros(s, dtype=torch.float32, device=dev)
