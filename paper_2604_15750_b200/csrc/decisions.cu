@@ -22,14 +22,14 @@ __device__ __forceinline__ float smooth_at(const float* x, int k, int n, int rad
   return __fdiv_rn(acc, (float)(hi - lo + 1));
 }
 
-// block-wide max / min over kThreads values (exact, order-free)
+// block-wide max / min over one value per thread (exact, order-free)
 __device__ __forceinline__ float block_max(float v, float* red) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   __syncthreads();
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   float t = red[0];
-  for (int i = 1; i < kThreads / 32; ++i) t = fmaxf(t, red[i]);
+  for (int i = 1; i < (int)(blockDim.x >> 5); ++i) t = fmaxf(t, red[i]);
   return t;
 }
 __device__ __forceinline__ int block_min_int(int v, int* red) {
@@ -38,7 +38,7 @@ __device__ __forceinline__ int block_min_int(int v, int* red) {
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   int t = red[0];
-  for (int i = 1; i < kThreads / 32; ++i) t = min(t, red[i]);
+  for (int i = 1; i < (int)(blockDim.x >> 5); ++i) t = min(t, red[i]);
   return t;
 }
 
@@ -125,17 +125,24 @@ __global__ void __launch_bounds__(kThreads) k_boundary(
   if (k == 0) block_len[b] = min(max(kstar, hp.L_min), Lw);
 }
 
+// one thread per window position, in whole warps (the block-wide reductions and scans cost a
+// barrier pair per warp-count step, so a window of 128 runs on 4 warps, not 8)
+static int boundary_threads(int max_window) {
+  const int t = (max_window + 31) / 32 * 32;
+  return t < 32 ? 32 : (t > kThreads ? kThreads : t);
+}
+
 void launch_boundary(const float* influence, const float* entropy, int ld, const SeqMeta& m,
                      const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
                      int32_t* block_len, cudaStream_t s) {
-  k_boundary<<<m.batch, kThreads, 0, s>>>(influence, entropy, ld, m, DevLens{}, hp, max_window, score,
+  k_boundary<<<m.batch, boundary_threads(max_window), 0, s>>>(influence, entropy, ld, m, DevLens{}, hp, max_window, score,
                                           cum_i, cum_s, block_len);
 }
 
 void launch_boundary_dev(const float* influence, const float* entropy, int ld, int batch, const DevLens& dl,
                          const Hyper& hp, int max_window, float* score, float* cum_i, float* cum_s,
                          int32_t* block_len, cudaStream_t s) {
-  k_boundary<<<batch, kThreads, 0, s>>>(influence, entropy, ld, SeqMeta{}, dl, hp, max_window, score,
+  k_boundary<<<batch, boundary_threads(max_window), 0, s>>>(influence, entropy, ld, SeqMeta{}, dl, hp, max_window, score,
                                         cum_i, cum_s, block_len);
 }
 
