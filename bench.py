@@ -597,7 +597,7 @@ def main():
     att_bytes = sum(n_layers * 2.0 * (P + nv * Rcap) * nkv_b for P in lens["ctx_len"])
     att_flops = sum(4.0 * n_layers * wl.n_q_heads * wl.head_dim * nv * Rcap * (P + Rcap) for P in lens["ctx_len"])
     rooflines = [roof,
-                 roof_entry("k_attn: bidirectional block attention, context K / V staged once for both variants",
+                 roof_entry("k_attn_tc: bidirectional block attention (one CTA per query tile; row tiles of 64 rows or fewer carry both variants over one staged context)",
                             stage_ms["attn"], att_bytes, att_flops, launches.get("attn", 0)),
                  roof_entry("k_lmhead_tc + k_lm_combine: LM head with streaming softmax / entropy / KL",
                             stage_ms["lmhead"], 2.0 * wl.vocab * wl.d_model,
